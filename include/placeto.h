@@ -1,0 +1,233 @@
+/*
+ * placeto.h - C ABI of the B200 (sm_100a) library for the Placeto policy forward.
+ *
+ * The library evaluates, for one computation DAG and a batch of B placement
+ * states, the graph-embedding policy network of Placeto (arXiv 1906.08879,
+ * Sec. 2.2 and Appendix A.7):
+ *
+ *   step 1  raw features per node and state                (Sec. 2.1, Sec. 2.2 step 1)
+ *   step 2  top-down and bottom-up message passing,
+ *           h_v = g( sum_{u in nbr(v)} f([h_u || x_u]) )    (Sec. 2.2 step 2)
+ *   step 3  pooling over the nodes that can reach the current node, that it
+ *           can reach, and the rest: h_i( sum l_i(e_u) )    (Sec. 2.2 step 3)
+ *   head    two-layer feed-forward net + softmax over the m devices (Appendix A.7)
+ *
+ * Conventions
+ *   - Pointers are marked HOST or DEVICE. All DEVICE pointers must be 16-byte
+ *     aligned and belong to the device that was current at placeto_graph_create.
+ *   - The caller owns every buffer (inputs, outputs, weights, workspace); the
+ *     library owns only placeto_graph objects. Forward calls allocate nothing,
+ *     do not synchronise (except the _host variant, see there) and run
+ *     asynchronously on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream). Two calls may run concurrently if their workspaces and
+ *     outputs are distinct.
+ *   - Every call returns a placeto_status. Problems the host can see (null or
+ *     misaligned pointers, sizes out of range, networks whose dimensions do not
+ *     fit d, F, m, a workspace that is too small, a graph with a cycle) are
+ *     rejected before any launch and leave the outputs untouched. CUDA launch
+ *     failures map to PLACETO_ERR_CUDA. Nothing aborts or traps.
+ *   - Node ids in all tensors are the caller's ids. Layouts are row-major:
+ *     X[n][B][F], H[n][B][d], logits/probs[B][m], dev/placed[B][n].
+ *   - Arithmetic is fp32. The order of the sums over neighbours and sets is
+ *     unspecified but fixed: a call is run-to-run deterministic for fixed
+ *     arguments and flags.
+ */
+#ifndef PLACETO_H_
+#define PLACETO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PLACETO_OK = 0,
+    PLACETO_ERR_INVALID_ARG = 1, /* null/misaligned pointer, size or dimension out of range */
+    PLACETO_ERR_NOT_DAG = 2,     /* cycle, self-loop or node id out of range */
+    PLACETO_ERR_WORKSPACE = 3,   /* workspace smaller than placeto_workspace_bytes() */
+    PLACETO_ERR_UNSUPPORTED = 4, /* dimensions beyond the limits below, or flag not applicable */
+    PLACETO_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
+    PLACETO_ERR_NO_MEMORY = 6    /* host or device allocation failed in graph_create */
+} placeto_status;
+
+/* Limits of this build. */
+#define PLACETO_MAX_D 128      /* embedding width d */
+#define PLACETO_MAX_F 64       /* feature width F */
+#define PLACETO_MAX_M 60       /* devices m (F = m + 4 in build_features) */
+#define PLACETO_MAX_HIDDEN 1024/* hidden width of any network */
+#define PLACETO_MAX_NODES 16384
+
+/* Human-readable name of a status (static string, never NULL). */
+const char *placeto_status_string(placeto_status s);
+
+/* ------------------------------------------------------------------ graph -- */
+
+typedef struct placeto_graph placeto_graph; /* opaque, library-owned */
+
+/* placeto_graph_create flags */
+#define PLACETO_GRAPH_DEVICE 0u    /* build on the host and upload to the current device */
+#define PLACETO_GRAPH_HOST_ONLY 1u /* build the host plan only (no CUDA call; forward calls
+                                      on such a graph return PLACETO_ERR_INVALID_ARG) */
+
+/*
+ * Builds the static plan of a DAG G(V, E) (Sec. 2: nodes are op groups, edges
+ * data dependencies u -> v) from a HOST edge list in any order:
+ *   - checks ids and acyclicity (PLACETO_ERR_NOT_DAG), drops repeated edges
+ *     (neighbours are sets);
+ *   - top-down levels (longest path from a root) and bottom-up levels (longest
+ *     path to a leaf), nodes bucketed by level, with the parent (resp. child)
+ *     lists in CSR form in level order: the schedule of step 2;
+ *   - the relation of every pair (c, u): u can reach c / c can reach u /
+ *     neither / same node: the three sets of step 3.
+ * src, dst: HOST int32[n_edges] (may be NULL when n_edges == 0). n >= 1.
+ * On success *out owns host and (unless HOST_ONLY) device copies of the plan;
+ * release it with placeto_graph_destroy. On failure *out is NULL.
+ */
+placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *src,
+                                    const int32_t *dst, uint32_t flags, placeto_graph **out);
+
+/* Sizes of the plan. Any output pointer may be NULL. n_edges counts distinct edges. */
+placeto_status placeto_graph_info(const placeto_graph *g, int32_t *n, int64_t *n_edges,
+                                  int32_t *n_levels_down, int32_t *n_levels_up,
+                                  int32_t *max_level_width);
+
+/*
+ * Read-only HOST view of the plan, valid until placeto_graph_destroy; meant
+ * for inspection and tests. dir 0 = top-down (neighbours are parents), 1 =
+ * bottom-up (neighbours are children).
+ *   level_ptr[n_levels+1] : positions of each level's nodes in `order`
+ *   order[n]              : node ids sorted by level, ascending id inside a level
+ *   nbr_ptr[n+1], nbr[]   : neighbour ids of order[p] are nbr[nbr_ptr[p] .. nbr_ptr[p+1]), ascending
+ *   relation[n*n]         : relation[c*n+u] = 0 u can reach c, 1 c can reach u, 2 neither, 3 u == c
+ */
+typedef struct {
+    int32_t n_levels;
+    const int32_t *level_ptr, *order, *nbr_ptr, *nbr;
+} placeto_level_view;
+placeto_status placeto_graph_host_view(const placeto_graph *g, placeto_level_view *down,
+                                       placeto_level_view *up, const uint8_t **relation);
+
+/* Releases the plan (device memory is freed with the creating device current). NULL is a no-op. */
+void placeto_graph_destroy(placeto_graph *g);
+
+/* ---------------------------------------------------------------- weights -- */
+
+/* One feed-forward network (Appendix A.7): y = act(v W1 + b1), then for two
+ * layers y = y W2 + b2; the activation also follows the last layer when
+ * final_act is 1. W row-major [in][out]. Pointers are DEVICE float arrays
+ * (W2, b2 NULL for one layer). */
+typedef struct {
+    int32_t n_layers;                     /* 1 or 2 */
+    int32_t in_dim, hidden_dim, out_dim;  /* hidden_dim ignored for one layer */
+    const float *W1, *b1, *W2, *b2;
+    int32_t act;                          /* 0 relu, 1 identity */
+    int32_t final_act;                    /* 0 or 1 */
+} placeto_mlp;
+
+/* All networks of the policy. f: (d+F) -> d and g: d -> d per direction
+ * (separate parameters, shared by all nodes of the direction); l[i]: (2d+F) -> d
+ * and h[i]: d -> d for i = 0 parents set, 1 children set, 2 parallel set;
+ * head: (5d+F) -> hidden -> m, normally with final_act = 0. */
+typedef struct {
+    int32_t d, F, m;
+    placeto_mlp f_down, g_down, f_up, g_up;
+    placeto_mlp l[3], h[3];
+    placeto_mlp head;
+} placeto_weights;
+
+/* ------------------------------------------------------------------ calls -- */
+
+/* Schedule of step 2 (the result does not depend on it beyond rounding order). */
+#define PLACETO_AUTO 0u        /* library picks */
+#define PLACETO_PER_LEVEL 1u   /* one launch per topological level */
+#define PLACETO_SLICED 2u      /* persistent: each thread block owns a slice of the state batch
+                                  and walks all levels, synchronising only inside the block
+                                  (states never interact) */
+#define PLACETO_COOPERATIVE 4u /* persistent cooperative launch: a level's nodes are spread over
+                                  blocks, grid-wide sync between levels (small B, wide levels) */
+#define PLACETO_GENERIC 8u     /* use only the dimension-generic kernels (no specialised ones) */
+
+typedef enum {
+    PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */
+    PLACETO_CALL_LOGITS = 1,      /* placeto_policy_logits */
+    PLACETO_CALL_FORWARD = 2,     /* placeto_policy_forward */
+    PLACETO_CALL_FORWARD_HOST = 3 /* placeto_policy_forward_host */
+} placeto_call;
+
+/* Bytes of DEVICE workspace `call` needs for batch size B (0 on invalid arguments).
+ * The workspace holds the per-node messages of step 2, partial sums of step 3 and,
+ * for the two policy_forward calls, the intermediate tensors X, H_down, H_up
+ * (plus the staged inputs and results for the _host call). */
+size_t placeto_workspace_bytes(const placeto_graph *g, const placeto_weights *w, int32_t B,
+                               placeto_call call, uint32_t flags);
+
+/*
+ * Step 1 (Sec. 2.1; Sec. 2.2 step 1): X[v][b] = [cost_v, bytes_v, one-hot_m(dev[b][v]),
+ * 1[v == cur[b]], placed[b][v] != 0], F = m + 4.
+ * cost, bytes: DEVICE float[n]; dev, placed: DEVICE uint8[B][n] (dev values < m; a larger
+ * value yields an all-zero one-hot); cur: DEVICE int32[B]; X: DEVICE float[n][B][m+4] (out).
+ */
+placeto_status placeto_build_features(const placeto_graph *g, const float *cost,
+                                      const float *bytes, const uint8_t *dev, const int32_t *cur,
+                                      const uint8_t *placed, int32_t m, int32_t B, float *X,
+                                      void *stream);
+
+/*
+ * Step 2 (Sec. 2.2 step 2), one progressive sweep per direction in topological
+ * order: h_v = g( sum_{u in nbr(v)} f([h_u || x_u]) ), nbr = parents for H_down,
+ * children for H_up; an empty neighbour set sums to zero. Uses w->f_*, w->g_*, w->d, w->F.
+ * X: DEVICE float[n][B][F] (in); H_down, H_up: DEVICE float[n][B][d] (out).
+ * workspace: DEVICE, at least placeto_workspace_bytes(.., PLACETO_CALL_EMBED, flags).
+ */
+placeto_status placeto_embed_forward(const placeto_graph *g, const placeto_weights *w,
+                                     const float *X, int32_t B, float *H_down, float *H_up,
+                                     void *workspace, size_t workspace_bytes, uint32_t flags,
+                                     void *stream);
+
+/*
+ * Step 3 and the head (Sec. 2.2 step 3, Appendix A.7). With e_u = [h_down_u || h_up_u || x_u]
+ * and c = cur[b]: a_i = h_i( sum_{u in S_i(c)} l_i(e_u) ) for the three sets (an empty set
+ * sums to zero), z = [e_c || a_0 || a_1 || a_2], logits = head(z), probs = softmax(logits)
+ * (max-subtracted). cur is authoritative for the sets; it is not re-derived from X.
+ * cur: DEVICE int32[B], each in [0, n) (a value out of range makes that state's outputs NaN);
+ * logits: DEVICE float[B][m] (out); probs: DEVICE float[B][m] (out) or NULL.
+ */
+placeto_status placeto_policy_logits(const placeto_graph *g, const placeto_weights *w,
+                                     const float *X, const float *H_down, const float *H_up,
+                                     const int32_t *cur, int32_t B, float *logits, float *probs,
+                                     void *workspace, size_t workspace_bytes, uint32_t flags,
+                                     void *stream);
+
+/*
+ * Whole path on DEVICE state arrays: steps 1-3 and the head; X and H live in the
+ * workspace. Arguments as in placeto_build_features and placeto_policy_logits
+ * (w->F must equal w->m + 4).
+ */
+placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weights *w,
+                                      const float *cost, const float *bytes, const uint8_t *dev,
+                                      const int32_t *cur, const uint8_t *placed, int32_t B,
+                                      float *logits, float *probs, void *workspace,
+                                      size_t workspace_bytes, uint32_t flags, void *stream);
+
+/*
+ * Whole path from HOST state arrays to HOST results: copies cost, bytes, dev, cur,
+ * placed to the device (cudaMemcpyAsync on `stream`; pinned host memory makes them
+ * truly asynchronous), runs the path, copies logits (and probs unless NULL) back and
+ * waits for the stream before returning. Weights and workspace stay DEVICE pointers.
+ */
+placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto_weights *w,
+                                           const float *cost, const float *bytes,
+                                           const uint8_t *dev, const int32_t *cur,
+                                           const uint8_t *placed, int32_t B, float *logits,
+                                           float *probs, void *workspace, size_t workspace_bytes,
+                                           uint32_t flags, void *stream);
+
+/* Number of kernels the most recent forward call of this thread launched (for accounting). */
+int32_t placeto_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PLACETO_H_ */

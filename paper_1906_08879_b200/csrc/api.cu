@@ -1,0 +1,438 @@
+// C ABI of the library (see include/placeto.h): argument validation, workspace
+// layout, schedule selection and kernel launches. No arithmetic of the policy
+// happens on the host.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "kernels.cuh"
+#include "plan.h"
+
+using namespace placeto;
+
+struct placeto_graph {
+    HostPlan host;
+    bool on_device = false;
+    int device = -1;
+    DeviceInfo info{};
+    int *d_ints = nullptr;       // one allocation for all int arrays
+    uint8_t *d_relation = nullptr;
+    DevLevels lv[2]{};
+};
+
+namespace placeto {
+
+static thread_local int t_launches = 0;
+void count_launch(int k) { t_launches += k; }
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool mlp_ok(const placeto_mlp &m, int in, int out) {
+    if (m.n_layers != 1 && m.n_layers != 2) return false;
+    if (m.in_dim != in || m.out_dim != out) return false;
+    if (m.act != 0 && m.act != 1) return false;
+    if (m.final_act != 0 && m.final_act != 1) return false;
+    if (!m.W1 || !m.b1 || !aligned16(m.W1) || !aligned16(m.b1)) return false;
+    if (m.n_layers == 2) {
+        if (m.hidden_dim < 1 || m.hidden_dim > PLACETO_MAX_HIDDEN) return false;
+        if (!m.W2 || !m.b2 || !aligned16(m.W2) || !aligned16(m.b2)) return false;
+    }
+    return true;
+}
+
+placeto_status dims_ok(const placeto_weights *w) {
+    if (!w) return PLACETO_ERR_INVALID_ARG;
+    if (w->d < 1 || w->F < 1 || w->m < 1) return PLACETO_ERR_INVALID_ARG;
+    if (w->d > PLACETO_MAX_D || w->F > PLACETO_MAX_F || w->m > PLACETO_MAX_M + 4) // head width
+        return PLACETO_ERR_UNSUPPORTED;
+    return PLACETO_OK;
+}
+
+placeto_status embed_weights_ok(const placeto_weights *w) {
+    placeto_status s = dims_ok(w);
+    if (s != PLACETO_OK) return s;
+    const int d = w->d, F = w->F;
+    if (!mlp_ok(w->f_down, d + F, d) || !mlp_ok(w->f_up, d + F, d) || !mlp_ok(w->g_down, d, d) ||
+        !mlp_ok(w->g_up, d, d))
+        return PLACETO_ERR_INVALID_ARG;
+    return PLACETO_OK;
+}
+
+placeto_status pool_weights_ok(const placeto_weights *w) {
+    placeto_status s = dims_ok(w);
+    if (s != PLACETO_OK) return s;
+    const int d = w->d, F = w->F;
+    for (int i = 0; i < 3; ++i)
+        if (!mlp_ok(w->l[i], 2 * d + F, d) || !mlp_ok(w->h[i], d, d)) return PLACETO_ERR_INVALID_ARG;
+    if (!mlp_ok(w->head, 5 * d + F, w->m)) return PLACETO_ERR_INVALID_ARG;
+    return PLACETO_OK;
+}
+
+struct Layout {
+    size_t msg[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
+    int chunks, chunk_nodes;
+};
+
+// Workspace layout shared by every call; a call uses the leading part it needs.
+Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, placeto_call call) {
+    Layout L{};
+    const size_t n = (size_t)g->host.n, d = (size_t)w->d, F = (size_t)w->F, m = (size_t)w->m;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    int chunks = pool_chunks((int)n, B, g->info);
+    L.chunk_nodes = ((int)n + chunks - 1) / chunks;
+    L.chunks = ((int)n + L.chunk_nodes - 1) / L.chunk_nodes;
+    if (call == PLACETO_CALL_EMBED || call >= PLACETO_CALL_FORWARD) {
+        L.msg[0] = take(n * B * d * sizeof(float));
+        L.msg[1] = take(n * B * d * sizeof(float));
+    }
+    if (call == PLACETO_CALL_LOGITS || call >= PLACETO_CALL_FORWARD)
+        L.partial = take((size_t)L.chunks * B * 3 * d * sizeof(float));
+    if (call >= PLACETO_CALL_FORWARD) {
+        L.X = take(n * B * F * sizeof(float));
+        L.H[0] = take(n * B * d * sizeof(float));
+        L.H[1] = take(n * B * d * sizeof(float));
+    }
+    if (call == PLACETO_CALL_FORWARD_HOST) {
+        L.cost = take(n * sizeof(float));
+        L.bytes = take(n * sizeof(float));
+        L.dev = take(n * B);
+        L.placed = take(n * B);
+        L.cur = take((size_t)B * sizeof(int32_t));
+        L.logits = take((size_t)B * m * sizeof(float));
+        L.probs = take((size_t)B * m * sizeof(float));
+    }
+    L.total = off;
+    return L;
+}
+
+unsigned pick_schedule(unsigned flags) {
+    if (flags & PLACETO_PER_LEVEL) return PLACETO_PER_LEVEL;
+    if (flags & PLACETO_COOPERATIVE) return PLACETO_COOPERATIVE;
+    return PLACETO_SLICED;
+}
+
+bool flags_ok(uint32_t flags) {
+    const uint32_t known = PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE | PLACETO_GENERIC;
+    if (flags & ~known) return false;
+    const uint32_t sched = flags & (PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE);
+    return (sched & (sched - 1)) == 0;   // at most one schedule
+}
+
+placeto_status cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return PLACETO_OK;
+    if (e == cudaErrorCooperativeLaunchTooLarge) return PLACETO_ERR_UNSUPPORTED;
+    return PLACETO_ERR_CUDA;
+}
+
+placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const float *X, int B,
+                         float *H_down, float *H_up, char *ws, const Layout &L, uint32_t flags,
+                         cudaStream_t stream) {
+    EmbedArgs a;
+    a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
+    a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
+    a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
+    a.X = X;
+    a.H[0] = H_down; a.H[1] = H_up;
+    a.M[0] = reinterpret_cast<float *>(ws + L.msg[0]);
+    a.M[1] = reinterpret_cast<float *>(ws + L.msg[1]);
+    a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
+    return cuda_status(launch_embed_generic(a, g->info, pick_schedule(flags), stream));
+}
+
+placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const float *X,
+                        const float *H_down, const float *H_up, const int32_t *cur, int B,
+                        float *logits, float *probs, char *ws, const Layout &L, uint32_t flags,
+                        cudaStream_t stream) {
+    (void)flags;
+    PoolArgs a;
+    for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
+    a.head = to_dev(w->head);
+    a.X = X; a.H[0] = H_down; a.H[1] = H_up;
+    a.cur = cur;
+    a.relation = g->d_relation;
+    a.partial = reinterpret_cast<float *>(ws + L.partial);
+    a.logits = logits; a.probs = probs;
+    a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d; a.m = w->m;
+    a.chunks = L.chunks; a.chunk_nodes = L.chunk_nodes;
+    return cuda_status(launch_policy_generic(a, g->info, stream));
+}
+
+placeto_status common_checks(const placeto_graph *g, int32_t B, const void *ws, size_t ws_bytes,
+                             size_t need, uint32_t flags) {
+    if (!g || !g->on_device || B < 1 || !flags_ok(flags)) return PLACETO_ERR_INVALID_ARG;
+    if ((size_t)B * g->host.n > (size_t)1 << 31) return PLACETO_ERR_UNSUPPORTED;
+    if (!ws || !aligned16(ws)) return PLACETO_ERR_INVALID_ARG;
+    if (ws_bytes < need) return PLACETO_ERR_WORKSPACE;
+    return PLACETO_OK;
+}
+
+}  // namespace
+}  // namespace placeto
+
+extern "C" {
+
+const char *placeto_status_string(placeto_status s) {
+    switch (s) {
+        case PLACETO_OK: return "ok";
+        case PLACETO_ERR_INVALID_ARG: return "invalid argument";
+        case PLACETO_ERR_NOT_DAG: return "edge list is not a DAG over [0, n)";
+        case PLACETO_ERR_WORKSPACE: return "workspace too small";
+        case PLACETO_ERR_UNSUPPORTED: return "unsupported dimensions or flag";
+        case PLACETO_ERR_CUDA: return "CUDA error";
+        case PLACETO_ERR_NO_MEMORY: return "out of memory";
+    }
+    return "unknown status";
+}
+
+placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *src,
+                                    const int32_t *dst, uint32_t flags, placeto_graph **out) {
+    if (!out) return PLACETO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (flags & ~PLACETO_GRAPH_HOST_ONLY) return PLACETO_ERR_INVALID_ARG;
+    placeto_graph *g = new (std::nothrow) placeto_graph();
+    if (!g) return PLACETO_ERR_NO_MEMORY;
+    placeto_status s = build_plan(n, n_edges, src, dst, g->host);
+    if (s != PLACETO_OK) { delete g; return s; }
+    if (flags & PLACETO_GRAPH_HOST_ONLY) { *out = g; return PLACETO_OK; }
+
+    auto fail = [&](placeto_status st) {
+        if (g->d_ints) cudaFree(g->d_ints);
+        if (g->d_relation) cudaFree(g->d_relation);
+        delete g;
+        return st;
+    };
+    if (cudaGetDevice(&g->device) != cudaSuccess) return fail(PLACETO_ERR_CUDA);
+    if (cudaDeviceGetAttribute(&g->info.sm_count, cudaDevAttrMultiProcessorCount, g->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&g->info.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, g->device) != cudaSuccess)
+        return fail(PLACETO_ERR_CUDA);
+    // one int allocation: per direction level_ptr, order, nbr_ptr, nbr (each padded to 4 ints)
+    size_t total = 0;
+    size_t offs[2][4];
+    for (int dir = 0; dir < 2; ++dir) {
+        const LevelPlan &p = g->host.dir[dir];
+        const size_t sizes[4] = {p.level_ptr.size(), p.order.size(), p.nbr_ptr.size(), p.nbr.size()};
+        for (int k = 0; k < 4; ++k) { offs[dir][k] = total; total += (sizes[k] + 3) & ~size_t(3); }
+    }
+    if (cudaMalloc(&g->d_ints, std::max<size_t>(total, 4) * sizeof(int)) != cudaSuccess)
+        return fail(PLACETO_ERR_NO_MEMORY);
+    if (cudaMalloc(&g->d_relation, g->host.relation.size()) != cudaSuccess)
+        return fail(PLACETO_ERR_NO_MEMORY);
+    for (int dir = 0; dir < 2; ++dir) {
+        const LevelPlan &p = g->host.dir[dir];
+        const std::vector<int32_t> *vecs[4] = {&p.level_ptr, &p.order, &p.nbr_ptr, &p.nbr};
+        for (int k = 0; k < 4; ++k)
+            if (!vecs[k]->empty() &&
+                cudaMemcpy(g->d_ints + offs[dir][k], vecs[k]->data(), vecs[k]->size() * sizeof(int),
+                           cudaMemcpyHostToDevice) != cudaSuccess)
+                return fail(PLACETO_ERR_CUDA);
+        g->lv[dir].n_levels = p.n_levels;
+        g->lv[dir].level_ptr = g->d_ints + offs[dir][0];
+        g->lv[dir].order = g->d_ints + offs[dir][1];
+        g->lv[dir].nbr_ptr = g->d_ints + offs[dir][2];
+        g->lv[dir].nbr = g->d_ints + offs[dir][3];
+    }
+    if (cudaMemcpy(g->d_relation, g->host.relation.data(), g->host.relation.size(),
+                   cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(PLACETO_ERR_CUDA);
+    g->on_device = true;
+    *out = g;
+    return PLACETO_OK;
+}
+
+placeto_status placeto_graph_info(const placeto_graph *g, int32_t *n, int64_t *n_edges,
+                                  int32_t *n_levels_down, int32_t *n_levels_up,
+                                  int32_t *max_level_width) {
+    if (!g) return PLACETO_ERR_INVALID_ARG;
+    if (n) *n = g->host.n;
+    if (n_edges) *n_edges = g->host.n_edges;
+    if (n_levels_down) *n_levels_down = g->host.dir[0].n_levels;
+    if (n_levels_up) *n_levels_up = g->host.dir[1].n_levels;
+    if (max_level_width) *max_level_width = g->host.max_level_width;
+    return PLACETO_OK;
+}
+
+placeto_status placeto_graph_host_view(const placeto_graph *g, placeto_level_view *down,
+                                       placeto_level_view *up, const uint8_t **relation) {
+    if (!g) return PLACETO_ERR_INVALID_ARG;
+    placeto_level_view *views[2] = {down, up};
+    for (int dir = 0; dir < 2; ++dir) {
+        if (!views[dir]) continue;
+        const LevelPlan &p = g->host.dir[dir];
+        views[dir]->n_levels = p.n_levels;
+        views[dir]->level_ptr = p.level_ptr.data();
+        views[dir]->order = p.order.data();
+        views[dir]->nbr_ptr = p.nbr_ptr.data();
+        views[dir]->nbr = p.nbr.data();
+    }
+    if (relation) *relation = g->host.relation.data();
+    return PLACETO_OK;
+}
+
+void placeto_graph_destroy(placeto_graph *g) {
+    if (!g) return;
+    if (g->on_device) {
+        int prev = -1;
+        cudaGetDevice(&prev);
+        if (prev != g->device) cudaSetDevice(g->device);
+        cudaFree(g->d_ints);
+        cudaFree(g->d_relation);
+        if (prev != g->device && prev >= 0) cudaSetDevice(prev);
+    }
+    delete g;
+}
+
+size_t placeto_workspace_bytes(const placeto_graph *g, const placeto_weights *w, int32_t B,
+                               placeto_call call, uint32_t flags) {
+    if (!g || !w || B < 1 || !flags_ok(flags) || dims_ok(w) != PLACETO_OK) return 0;
+    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_FORWARD_HOST) return 0;
+    placeto_graph tmp_info;   // HOST_ONLY graphs have no device info: assume a full B200
+    const placeto_graph *use = g;
+    if (!g->on_device) {
+        tmp_info.host.n = g->host.n;
+        tmp_info.info.sm_count = 148;
+        tmp_info.info.max_smem_optin = 227 * 1024;
+        use = &tmp_info;
+    }
+    return std::max<size_t>(make_layout(use, w, B, call).total, kAlign);
+}
+
+placeto_status placeto_build_features(const placeto_graph *g, const float *cost,
+                                      const float *bytes, const uint8_t *dev, const int32_t *cur,
+                                      const uint8_t *placed, int32_t m, int32_t B, float *X,
+                                      void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device || B < 1 || m < 1 || m > PLACETO_MAX_M) return PLACETO_ERR_INVALID_ARG;
+    if (!cost || !bytes || !dev || !cur || !placed || !X) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(cur) ||
+        !aligned16(placed) || !aligned16(X))
+        return PLACETO_ERR_INVALID_ARG;
+    return cuda_status(launch_features(g->host.n, B, m, cost, bytes, dev, cur, placed, X,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+placeto_status placeto_embed_forward(const placeto_graph *g, const placeto_weights *w,
+                                     const float *X, int32_t B, float *H_down, float *H_up,
+                                     void *workspace, size_t workspace_bytes, uint32_t flags,
+                                     void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_EMBED);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, flags);
+    if (s != PLACETO_OK) return s;
+    if (!X || !H_down || !H_up || !aligned16(X) || !aligned16(H_down) || !aligned16(H_up))
+        return PLACETO_ERR_INVALID_ARG;
+    return run_embed(g, w, X, B, H_down, H_up, static_cast<char *>(workspace), L, flags,
+                     static_cast<cudaStream_t>(stream));
+}
+
+placeto_status placeto_policy_logits(const placeto_graph *g, const placeto_weights *w,
+                                     const float *X, const float *H_down, const float *H_up,
+                                     const int32_t *cur, int32_t B, float *logits, float *probs,
+                                     void *workspace, size_t workspace_bytes, uint32_t flags,
+                                     void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_LOGITS);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, flags);
+    if (s != PLACETO_OK) return s;
+    if (!X || !H_down || !H_up || !cur || !logits) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(H_down) || !aligned16(H_up) || !aligned16(cur) ||
+        !aligned16(logits) || (probs && !aligned16(probs)))
+        return PLACETO_ERR_INVALID_ARG;
+    return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, static_cast<char *>(workspace),
+                    L, flags, static_cast<cudaStream_t>(stream));
+}
+
+placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weights *w,
+                                      const float *cost, const float *bytes, const uint8_t *dev,
+                                      const int32_t *cur, const uint8_t *placed, int32_t B,
+                                      float *logits, float *probs, void *workspace,
+                                      size_t workspace_bytes, uint32_t flags, void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s == PLACETO_OK) s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1 || w->m > PLACETO_MAX_M || w->F != w->m + 4) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_FORWARD);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, flags);
+    if (s != PLACETO_OK) return s;
+    if (!cost || !bytes || !dev || !cur || !placed || !logits) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(cur) ||
+        !aligned16(placed) || !aligned16(logits) || (probs && !aligned16(probs)))
+        return PLACETO_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float *X = reinterpret_cast<float *>(ws + L.X);
+    float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
+    float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
+    s = cuda_status(launch_features(g->host.n, B, w->m, cost, bytes, dev, cur, placed, X, st));
+    if (s != PLACETO_OK) return s;
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st);
+    if (s != PLACETO_OK) return s;
+    return run_pool(g, w, X, Hd, Hu, cur, B, logits, probs, ws, L, flags, st);
+}
+
+placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto_weights *w,
+                                           const float *cost, const float *bytes,
+                                           const uint8_t *dev, const int32_t *cur,
+                                           const uint8_t *placed, int32_t B, float *logits,
+                                           float *probs, void *workspace, size_t workspace_bytes,
+                                           uint32_t flags, void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s == PLACETO_OK) s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1 || w->m > PLACETO_MAX_M || w->F != w->m + 4) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_FORWARD_HOST);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, flags);
+    if (s != PLACETO_OK) return s;
+    if (!cost || !bytes || !dev || !cur || !placed || !logits) return PLACETO_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t n = (size_t)g->host.n;
+    float *d_cost = reinterpret_cast<float *>(ws + L.cost);
+    float *d_bytes = reinterpret_cast<float *>(ws + L.bytes);
+    uint8_t *d_dev = reinterpret_cast<uint8_t *>(ws + L.dev);
+    uint8_t *d_placed = reinterpret_cast<uint8_t *>(ws + L.placed);
+    int32_t *d_cur = reinterpret_cast<int32_t *>(ws + L.cur);
+    float *d_logits = reinterpret_cast<float *>(ws + L.logits);
+    float *d_probs = reinterpret_cast<float *>(ws + L.probs);
+    const size_t mB = (size_t)B * w->m * sizeof(float);
+    if (cudaMemcpyAsync(d_cost, cost, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_bytes, bytes, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_dev, dev, n * B, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_placed, placed, n * B, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_cur, cur, (size_t)B * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PLACETO_ERR_CUDA;
+    float *X = reinterpret_cast<float *>(ws + L.X);
+    float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
+    float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
+    s = cuda_status(launch_features(g->host.n, B, w->m, d_cost, d_bytes, d_dev, d_cur, d_placed, X, st));
+    if (s != PLACETO_OK) return s;
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st);
+    if (s != PLACETO_OK) return s;
+    s = run_pool(g, w, X, Hd, Hu, d_cur, B, d_logits, probs ? d_probs : nullptr, ws, L, flags, st);
+    if (s != PLACETO_OK) return s;
+    if (cudaMemcpyAsync(logits, d_logits, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PLACETO_ERR_CUDA;
+    if (probs && cudaMemcpyAsync(probs, d_probs, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PLACETO_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+int32_t placeto_last_launch_count(void) { return t_launches; }
+
+}  // extern "C"

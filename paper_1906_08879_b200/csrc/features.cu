@@ -1,0 +1,64 @@
+// Step 1 of the policy (Sec. 2.1 and Sec. 2.2 step 1 of the Placeto paper):
+// raw per-node, per-state features
+//   x = [cost, bytes, one-hot(device), is-current, is-placed],  F = m + 4,
+// written as X[n][B][F]. The state arrays are state-major (dev[B][n]) while X
+// is node-major, so a block transposes a 32-node x 32-state tile through
+// shared memory: loads run along nodes, stores along (state, feature).
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kTile = 32;
+
+__global__ void __launch_bounds__(256)
+features_kernel(int n, int B, int m, const float *__restrict__ cost,
+                const float *__restrict__ bytes, const uint8_t *__restrict__ dev,
+                const int *__restrict__ cur, const uint8_t *__restrict__ placed,
+                float *__restrict__ X) {
+    __shared__ uint8_t s_dev[kTile][kTile + 4];
+    __shared__ uint8_t s_placed[kTile][kTile + 4];
+    __shared__ int s_cur[kTile];
+    const int v0 = blockIdx.x * kTile, b0 = blockIdx.y * kTile;
+    const int F = m + 4;
+    for (int i = threadIdx.x; i < kTile * kTile; i += blockDim.x) {
+        const int bl = i / kTile, vl = i % kTile;
+        const int b = b0 + bl, v = v0 + vl;
+        const bool ok = b < B && v < n;
+        s_dev[bl][vl] = ok ? dev[(size_t)b * n + v] : 0;
+        s_placed[bl][vl] = ok ? placed[(size_t)b * n + v] : 0;
+    }
+    if (threadIdx.x < kTile) s_cur[threadIdx.x] = (b0 + threadIdx.x < B) ? cur[b0 + threadIdx.x] : -1;
+    __syncthreads();
+    const int nb = min(kTile, B - b0);
+    const int nv = min(kTile, n - v0);
+    for (int vl = 0; vl < nv; ++vl) {
+        const int v = v0 + vl;
+        const float c = cost[v], s = bytes[v];
+        float *out = X + ((size_t)v * B + b0) * F;
+        for (int i = threadIdx.x; i < nb * F; i += blockDim.x) {
+            const int bl = i / F, k = i - bl * F;
+            float val;
+            if (k == 0) val = c;
+            else if (k == 1) val = s;
+            else if (k < 2 + m) val = (s_dev[bl][vl] == k - 2) ? 1.f : 0.f;
+            else if (k == 2 + m) val = (s_cur[bl] == v) ? 1.f : 0.f;
+            else val = s_placed[bl][vl] ? 1.f : 0.f;
+            out[i] = val;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
+                            const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
+                            cudaStream_t stream) {
+    dim3 grid((n + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+    features_kernel<<<grid, 256, 0, stream>>>(n, B, m, cost, bytes, dev, cur, placed, X);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace placeto

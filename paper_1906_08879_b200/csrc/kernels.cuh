@@ -1,0 +1,86 @@
+// Device-side argument structs and launcher declarations shared by the
+// library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstddef>
+#include <cstdint>
+
+#include "placeto.h"
+
+namespace placeto {
+
+// One direction's level schedule in device memory (see placeto_graph_host_view).
+struct DevLevels {
+    int n_levels;
+    const int *level_ptr, *order, *nbr_ptr, *nbr;
+};
+
+// One feed-forward network with device pointers.
+struct DevMlp {
+    int n_layers, in_dim, hidden_dim, out_dim, act, final_act;
+    const float *W1, *b1, *W2, *b2;
+};
+
+inline DevMlp to_dev(const placeto_mlp &m) {
+    DevMlp d;
+    d.n_layers = m.n_layers;
+    d.in_dim = m.in_dim;
+    d.hidden_dim = m.n_layers == 2 ? m.hidden_dim : m.out_dim;
+    d.out_dim = m.out_dim;
+    d.act = m.act;
+    d.final_act = m.final_act;
+    d.W1 = m.W1; d.b1 = m.b1; d.W2 = m.W2; d.b2 = m.b2;
+    return d;
+}
+
+// Floats a network occupies when staged contiguously (W1, b1, W2, b2).
+inline size_t mlp_floats(const DevMlp &m) {
+    size_t s = (size_t)m.in_dim * m.hidden_dim + m.hidden_dim;
+    if (m.n_layers == 2) s += (size_t)m.hidden_dim * m.out_dim + m.out_dim;
+    return s;
+}
+
+struct EmbedArgs {
+    DevLevels lv[2];
+    DevMlp f[2], g[2];
+    const float *X;
+    float *H[2];   // outputs [n][B][d]
+    float *M[2];   // messages f([h || x]) per node and state, [n][B][d] (workspace)
+    int n, B, F, d;
+};
+
+struct PoolArgs {
+    DevMlp l[3], h[3], head;
+    const float *X, *H[2];
+    const int *cur;
+    const uint8_t *relation;   // [n][n]
+    float *partial;            // [chunks][B][3][d] (workspace)
+    float *logits, *probs;     // [B][m]; probs may be null
+    int n, B, F, d, m;
+    int chunks, chunk_nodes;
+};
+
+struct DeviceInfo {
+    int sm_count;
+    int max_smem_optin;   // bytes per block
+};
+
+// Counts launches of the calling thread's current forward call.
+void count_launch(int k = 1);
+
+// features.cu
+cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
+                            const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
+                            cudaStream_t stream);
+
+// embed_generic.cu: dimension-generic message passing. schedule is one of
+// PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.
+cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,
+                                 cudaStream_t stream);
+
+// policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
+int pool_chunks(int n, int B, const DeviceInfo &di);
+cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
+
+}  // namespace placeto

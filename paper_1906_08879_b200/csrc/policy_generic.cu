@@ -1,0 +1,257 @@
+// Step 3 and the head of the policy (Sec. 2.2 step 3 and Appendix A.7 of the
+// Placeto paper), for any widths.
+//
+// With e_u = [h_down_u || h_up_u || x_u] and c the state's current node,
+//   a_i = h_i( sum_{u in S_i(c)} l_i(e_u) ),  i = can-reach-c / reachable-from-c / neither,
+//   logits = head([e_c || a_0 || a_1 || a_2]),  probs = softmax(logits).
+// Kernel 1 cuts the nodes into chunks and writes, per chunk and state, the three
+// partial sums of l_i(e_u) (one warp per state, lanes over the output columns,
+// the set of each node read from the relation row of c). Kernel 2 adds the
+// chunks in a fixed order (deterministic, no atomics), applies h_i, the head and
+// the softmax, one block per state.
+#include <algorithm>
+#include <cmath>
+
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kPoolThreads = 256;
+constexpr int kPoolWarps = kPoolThreads / 32;
+constexpr int kMaxCols = PLACETO_MAX_D / 32;   // output columns per lane
+constexpr int kHeadThreads = 128;
+
+struct PoolPlan {
+    int states_per_block;
+    int weights_in_smem;
+    int e_stride;       // floats of the per-warp row buffer (input row + hidden row)
+    size_t smem_bytes;
+};
+
+__global__ void __launch_bounds__(kPoolThreads)
+pool_partial_kernel(const PoolArgs a, const PoolPlan p) {
+    extern __shared__ __align__(16) float smem[];
+    const int d = a.d, F = a.F, n = a.n, B = a.B;
+    const int E = 2 * d + F;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // l_i weights: staged contiguously per set when they fit
+    const float *W1[3], *b1[3], *W2[3], *b2[3];
+    float *w = smem;
+    for (int i = 0; i < 3; ++i) {
+        W1[i] = a.l[i].W1; b1[i] = a.l[i].b1; W2[i] = a.l[i].W2; b2[i] = a.l[i].b2;
+        if (p.weights_in_smem) {
+            auto stage = [&](const float *src, size_t count) {
+                float *dst = w;
+                for (size_t k = threadIdx.x; k < count; k += blockDim.x) dst[k] = src[k];
+                w += (count + 3) & ~size_t(3);
+                return (const float *)dst;
+            };
+            W1[i] = stage(a.l[i].W1, (size_t)a.l[i].in_dim * a.l[i].hidden_dim);
+            b1[i] = stage(a.l[i].b1, a.l[i].hidden_dim);
+            if (a.l[i].n_layers == 2) {
+                W2[i] = stage(a.l[i].W2, (size_t)a.l[i].hidden_dim * a.l[i].out_dim);
+                b2[i] = stage(a.l[i].b2, a.l[i].out_dim);
+            }
+        }
+    }
+    float *row = w + (size_t)warp * p.e_stride;   // [E] input row, then hidden row
+    float *hid = row + ((E + 3) & ~3);
+    __syncthreads();
+
+    const int chunk = blockIdx.x;
+    const int u0 = chunk * a.chunk_nodes, u1 = min(n, u0 + a.chunk_nodes);
+    const int bs0 = blockIdx.y * p.states_per_block;
+    const int bs1 = min(B, bs0 + p.states_per_block);
+    for (int b = bs0 + warp; b < bs1; b += kPoolWarps) {
+        const int c = a.cur[b];
+        float acc[3][kMaxCols];
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+#pragma unroll
+            for (int t = 0; t < kMaxCols; ++t) acc[i][t] = 0.f;
+        const bool valid = c >= 0 && c < n;
+        if (valid) {
+            const uint8_t *rel = a.relation + (size_t)c * n;
+            for (int u = u0; u < u1; ++u) {
+                const int i = rel[u];
+                if (i == 3) continue;
+                const float *hd = a.H[0] + ((size_t)u * B + b) * d;
+                const float *hu = a.H[1] + ((size_t)u * B + b) * d;
+                const float *x = a.X + ((size_t)u * B + b) * F;
+                for (int k = lane; k < d; k += 32) { row[k] = hd[k]; row[d + k] = hu[k]; }
+                for (int k = lane; k < F; k += 32) row[2 * d + k] = x[k];
+                __syncwarp();
+                const DevMlp &net = a.l[i];
+                const bool relu = net.act == 0;
+                const float *in = row;
+                int in_dim = E;
+                const float *W = W1[i], *bias = b1[i];
+                if (net.n_layers == 2) {
+                    for (int j = lane; j < net.hidden_dim; j += 32) {
+                        float s = bias[j];
+                        for (int k = 0; k < E; ++k) s = fmaf(in[k], W[k * net.hidden_dim + j], s);
+                        hid[j] = relu ? fmaxf(s, 0.f) : s;
+                    }
+                    __syncwarp();
+                    in = hid; in_dim = net.hidden_dim; W = W2[i]; bias = b2[i];
+                }
+#pragma unroll
+                for (int t = 0; t < kMaxCols; ++t) {
+                    const int j = lane + 32 * t;
+                    if (j < d) {
+                        float s = bias[j];
+                        for (int k = 0; k < in_dim; ++k) s = fmaf(in[k], W[k * d + j], s);
+                        if (relu && net.final_act) s = fmaxf(s, 0.f);
+#pragma unroll
+                        for (int ii = 0; ii < 3; ++ii) acc[ii][t] += (ii == i) ? s : 0.f;
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        float *out = a.partial + ((size_t)chunk * B + b) * 3 * d;
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+#pragma unroll
+            for (int t = 0; t < kMaxCols; ++t) {
+                const int j = lane + 32 * t;
+                if (j < d) out[i * d + j] = valid ? acc[i][t] : nanf("");
+            }
+    }
+}
+
+// y[0..out) = act(bias + v W) with the whole block; v, y in shared memory.
+__device__ __forceinline__ void block_dense(const float *__restrict__ W,
+                                            const float *__restrict__ bias, int in, int out,
+                                            bool relu, const float *v, float *y) {
+    if (out >= 32) {
+        for (int j = threadIdx.x; j < out; j += blockDim.x) {
+            float s = bias[j];
+            for (int k = 0; k < in; ++k) s = fmaf(v[k], W[(size_t)k * out + j], s);
+            y[j] = relu ? fmaxf(s, 0.f) : s;
+        }
+    } else {
+        // few outputs (the device logits): one warp per output, lanes split the
+        // inner dimension and combine with a shuffle reduction
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+        for (int j = warp; j < out; j += nw) {
+            float s = 0.f;
+            for (int k = lane; k < in; k += 32) s = fmaf(v[k], W[(size_t)k * out + j], s);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            s += bias[j];
+            if (lane == 0) y[j] = relu ? fmaxf(s, 0.f) : s;
+        }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ float *block_mlp(const DevMlp &net, const float *in, float *tmp,
+                                            float *out) {
+    const bool relu = net.act == 0;
+    if (net.n_layers == 1) {
+        block_dense(net.W1, net.b1, net.in_dim, net.out_dim, relu && net.final_act, in, out);
+        return out;
+    }
+    block_dense(net.W1, net.b1, net.in_dim, net.hidden_dim, relu, in, tmp);
+    block_dense(net.W2, net.b2, net.hidden_dim, net.out_dim, relu && net.final_act, tmp, out);
+    return out;
+}
+
+__global__ void __launch_bounds__(kHeadThreads)
+pool_head_kernel(const PoolArgs a, int tmp_floats) {
+    extern __shared__ __align__(16) float smem[];
+    const int d = a.d, F = a.F, B = a.B, m = a.m;
+    const int E = 2 * d + F, Z = 5 * d + F;
+    float *z = smem;                      // [Z]
+    float *sum = z + ((Z + 3) & ~3);      // [3][d]
+    float *tmp = sum + 3 * d;             // [tmp_floats] hidden rows
+    float *lg = tmp + tmp_floats;         // [m]
+    const int b = blockIdx.x;
+    const int c = a.cur[b];
+    const bool valid = c >= 0 && c < a.n;
+    for (int j = threadIdx.x; j < 3 * d; j += blockDim.x) {
+        float s = 0.f;
+        for (int ch = 0; ch < a.chunks; ++ch) s += a.partial[((size_t)ch * B + b) * 3 * d + j];
+        sum[j] = s;
+    }
+    if (valid) {
+        for (int k = threadIdx.x; k < E; k += blockDim.x)
+            z[k] = k < d ? a.H[0][((size_t)c * B + b) * d + k]
+                 : k < 2 * d ? a.H[1][((size_t)c * B + b) * d + (k - d)]
+                             : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
+    } else {
+        for (int k = threadIdx.x; k < E; k += blockDim.x) z[k] = nanf("");
+    }
+    __syncthreads();
+    for (int i = 0; i < 3; ++i) block_mlp(a.h[i], sum + i * d, tmp, z + E + i * d);
+    block_mlp(a.head, z, tmp, lg);
+    if (threadIdx.x == 0) {
+        float mx = lg[0];
+        for (int k = 1; k < m; ++k) mx = fmaxf(mx, lg[k]);
+        float tot = 0.f;
+        for (int k = 0; k < m; ++k) tot += expf(lg[k] - mx);
+        for (int k = 0; k < m; ++k) {
+            // a current node out of range yields NaN (ReLU would swallow a NaN input)
+            a.logits[(size_t)b * m + k] = valid ? lg[k] : nanf("");
+            if (a.probs) a.probs[(size_t)b * m + k] = valid ? expf(lg[k] - mx) / tot : nanf("");
+        }
+    }
+}
+
+}  // namespace
+
+int pool_chunks(int n, int B, const DeviceInfo &di) {
+    // enough (chunk, state-group) blocks to fill the device a few times over
+    const int state_blocks = (B + kPoolWarps - 1) / kPoolWarps;
+    int chunks = (4 * di.sm_count + state_blocks - 1) / state_blocks;
+    chunks = std::max(1, std::min(chunks, (n + 7) / 8));
+    return chunks;
+}
+
+cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+    PoolPlan p;
+    const int E = 2 * a.d + a.F;
+    int max_hidden = 0;
+    size_t wfloats = 0;
+    for (int i = 0; i < 3; ++i) {
+        const DevMlp &m = a.l[i];
+        if (m.n_layers == 2) max_hidden = std::max(max_hidden, m.hidden_dim);
+        wfloats += (((size_t)m.in_dim * m.hidden_dim + 3) & ~size_t(3)) + ((m.hidden_dim + 3) & ~3);
+        if (m.n_layers == 2)
+            wfloats += (((size_t)m.hidden_dim * m.out_dim + 3) & ~size_t(3)) + ((m.out_dim + 3) & ~3);
+    }
+    p.e_stride = ((E + 3) & ~3) + ((max_hidden + 3) & ~3);
+    const size_t rows_bytes = (size_t)kPoolWarps * p.e_stride * sizeof(float);
+    const size_t budget = (size_t)std::min(di.max_smem_optin, 200 * 1024);
+    p.weights_in_smem = (wfloats * sizeof(float) + rows_bytes <= budget) ? 1 : 0;
+    p.smem_bytes = rows_bytes + (p.weights_in_smem ? wfloats * sizeof(float) : 0);
+    p.states_per_block = kPoolWarps;
+    cudaError_t err = cudaFuncSetAttribute(pool_partial_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)p.smem_bytes);
+    if (err != cudaSuccess) return err;
+    dim3 grid(a.chunks, (a.B + p.states_per_block - 1) / p.states_per_block);
+    pool_partial_kernel<<<grid, kPoolThreads, p.smem_bytes, stream>>>(a, p);
+    count_launch();
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+
+    const int Z = 5 * a.d + a.F;
+    int tmp_floats = a.head.n_layers == 2 ? a.head.hidden_dim : 0;
+    for (int i = 0; i < 3; ++i)
+        if (a.h[i].n_layers == 2) tmp_floats = std::max(tmp_floats, a.h[i].hidden_dim);
+    tmp_floats = (tmp_floats + 3) & ~3;
+    const size_t head_smem = (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m + 4) * sizeof(float);
+    err = cudaFuncSetAttribute(pool_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)head_smem);
+    if (err != cudaSuccess) return err;
+    pool_head_kernel<<<a.B, kHeadThreads, head_smem, stream>>>(a, tmp_floats);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace placeto

@@ -72,9 +72,9 @@ def closure(n, src, dst):
     A = np.zeros((n, n), dtype=bool)
     A[np.asarray(src, dtype=int), np.asarray(dst, dtype=int)] = True
     R = A.copy()
-    for _ in range(max(n, 1)):
-        R2 = R | ((R.astype(np.int64) @ A.astype(np.int64)) > 0)
+    while True:                       # paths of length <= 2^k after k squarings
+        Rf = R.astype(np.float32)
+        R2 = R | ((Rf @ Rf) > 0)
         if (R2 == R).all():
-            break
+            return R
         R = R2
-    return R

@@ -1,0 +1,309 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU
+checker on the same seeded inputs, element by element.
+
+Tolerances (fp32 path): for every output row (the d-vector of one node and
+state, or the m logits of one state)
+    max_i |gpu_i - ref_i| / max(|ref_i|, 0.1 * ||ref row||_inf)  <= 1e-4
+and, normwise,
+    max_i |gpu_i - ref_i| / ||ref row||_inf                      <= 2e-5.
+The device argmax must equal the checker's wherever the checker's top-2 logit
+gap exceeds max(1e-3, 2e-5 * ||logits||_inf) (the second term is the normwise
+tolerance: below it fp32 cannot resolve the order at the raw feature scale).
+"""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import paper_1906_08879_b200 as placeto
+from gen import configs, states
+from oracle import oracle
+from tests.helpers import net, random_dag, rng, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL_ELEM, TOL_NORM = 1e-4, 2e-5
+SCHEDULES = {"sliced": placeto.PLACETO_SLICED, "per_level": placeto.PLACETO_PER_LEVEL,
+             "cooperative": placeto.PLACETO_COOPERATIVE}
+
+
+def dev_t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def assert_close(got, ref, what):
+    got = got.detach().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.isfinite(got).all(), what
+    e1 = row_rel_err(got, ref, 0.1)
+    e2 = row_rel_err(got, ref, 1.0)
+    assert e1 <= TOL_ELEM and e2 <= TOL_NORM, "%s: elementwise %.3g normwise %.3g" % (what, e1, e2)
+
+
+def assert_argmax(logits, ref_logits):
+    logits = logits.detach().cpu().numpy()
+    srt = np.sort(ref_logits, axis=1)
+    gap = srt[:, -1] - srt[:, -2] if ref_logits.shape[1] > 1 else np.full(len(srt), np.inf)
+    need = gap > np.maximum(1e-3, TOL_NORM * np.abs(ref_logits).max(axis=1))
+    same = logits.argmax(axis=1) == ref_logits.argmax(axis=1)
+    assert same[need].all(), "argmax differs on %d decisive states" % int((~same[need]).sum())
+    return int(need.sum())
+
+
+def gpu_forward(cfg, flags=0, sel=None):
+    """features -> embed -> logits through the three C entry points."""
+    devs, cur, placed = cfg["dev"], cfg["cur"], cfg["placed"]
+    if sel is not None:
+        devs, cur, placed = devs[sel], cur[sel], placed[sel]
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    cur_d = dev_t(cur)
+    X = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(devs),
+                                       cur_d, dev_t(placed), cfg["m"])
+    Hd, Hu = placeto.placeto_embed_forward(g, w, X, flags=flags)
+    logits, probs = placeto.placeto_policy_logits(g, w, X, Hd, Hu, cur_d, flags=flags)
+    torch.cuda.synchronize()
+    return {"X": X, "H_down": Hd, "H_up": Hu, "logits": logits, "probs": probs, "graph": g, "w": w}
+
+
+def compare(cfg, out, ref, sel=None):
+    pick = (lambda t: t) if sel is None else (lambda t: t[:, sel])
+    np.testing.assert_array_equal(pick(out["X"]).cpu().numpy(), ref["X"].astype(np.float32))
+    assert_close(pick(out["H_down"]), ref["H_down"], "H_down")
+    assert_close(pick(out["H_up"]), ref["H_up"], "H_up")
+    lg = out["logits"] if sel is None else out["logits"][sel]
+    pr = out["probs"] if sel is None else out["probs"][sel]
+    assert_close(lg, ref["logits"], "logits")
+    assert_argmax(lg, ref["logits"])
+    p = pr.cpu().numpy()
+    np.testing.assert_allclose(p.sum(axis=1), 1.0, rtol=1e-5)
+    # probabilities follow the logits: compare against the softmax of the device logits
+    l64 = lg.cpu().numpy().astype(np.float64)
+    sm = np.exp(l64 - l64.max(axis=1, keepdims=True))
+    sm /= sm.sum(axis=1, keepdims=True)
+    np.testing.assert_allclose(p, sm, atol=2e-6)
+    # and the checker's where the logit error cannot move them
+    scale = np.abs(ref["logits"]).max(axis=1)
+    calm = scale < 50.0
+    if calm.any():
+        np.testing.assert_allclose(p[calm], ref["probs"][calm], atol=5e-4)
+
+
+# ------------------------------------------------------------ the configs ---
+
+@pytest.mark.parametrize("schedule", list(SCHEDULES))
+@pytest.mark.parametrize("normalise", [False, True])
+def test_tiny(schedule, normalise):
+    cfg = configs.make("tiny", normalise=normalise)
+    out = gpu_forward(cfg, SCHEDULES[schedule])
+    compare(cfg, out, oracle.forward(cfg))
+
+
+@pytest.mark.parametrize("schedule", list(SCHEDULES))
+def test_inception(schedule):
+    cfg = configs.make("inception")
+    out = gpu_forward(cfg, SCHEDULES[schedule])
+    compare(cfg, out, oracle.forward(cfg, threads=8))
+
+
+def test_inception_normalised():
+    cfg = configs.make("inception", normalise=True)
+    compare(cfg, gpu_forward(cfg), oracle.forward(cfg, threads=8))
+
+
+@pytest.mark.parametrize("normalise", [False, True])
+def test_nmt(normalise):
+    cfg = configs.make("nmt", normalise=normalise)
+    out = gpu_forward(cfg)
+    compare(cfg, out, oracle.forward(cfg, threads=8))
+
+
+def test_nasnet_full_batch_sampled_states():
+    """Full size on the GPU (n ~ 2100, B = 512, d = 64); the checker evaluates
+    a sample of states one by one (states are independent)."""
+    cfg = configs.make("nasnet")
+    out = gpu_forward(cfg)
+    sel = np.asarray([0, 1, 63, 64, 255, 256, 300, 448, 510, 511])
+    compare(cfg, out, oracle.forward(cfg, threads=8, states=sel), sel=sel)
+    for k in ("H_down", "H_up", "logits", "probs"):
+        assert torch.isfinite(out[k]).all()
+
+
+@pytest.mark.parametrize("i", [0, 1, 30, 63])
+def test_episode_sweep(i):
+    cfg = configs.make_sweep(i)
+    out = gpu_forward(cfg)
+    n = cfg["n"]
+    sel = None if n <= 320 else np.unique(np.linspace(0, n - 1, 48).astype(int))
+    ref = oracle.forward(cfg, threads=8, states=sel)
+    compare(cfg, out, ref, sel=sel)
+
+
+# ------------------------------------------------------------- edge cases ---
+
+def _small_case(n, src, dst, d=8, m=3, B=5, layers=2, act=0, seed=0, schedule=0, F=None):
+    r = rng(seed)
+    F_ = m + 4
+    cfg = {"n": n, "src": np.asarray(src, np.int32), "dst": np.asarray(dst, np.int32), "m": m,
+           "d": d, "F": F_}
+    cfg["cost"], cfg["bytes"] = states.node_costs(r, n, normalise=True)
+    cfg["dev"], cfg["cur"], cfg["placed"] = states.random_states(r, n, m, B)
+    cfg["weights"] = states.policy_weights(r, d, F_, m, layers, act, 0.1)
+    out = gpu_forward(cfg, schedule)
+    compare(cfg, out, oracle.forward(cfg))
+
+
+@pytest.mark.parametrize("schedule", list(SCHEDULES))
+def test_degenerate_graphs(schedule):
+    s = SCHEDULES[schedule]
+    e = np.zeros(0, np.int32)
+    _small_case(1, e, e, schedule=s)                                   # one node
+    _small_case(5, e, e, schedule=s)                                   # no edges
+    _small_case(9, np.arange(8), np.arange(1, 9), schedule=s)          # chain
+    _small_case(7, np.zeros(6, np.int32), np.arange(1, 7), schedule=s) # star out
+    _small_case(7, np.arange(1, 7), np.zeros(6, np.int32), schedule=s) # star in (fan-in 6)
+    _small_case(4, [0, 0, 1, 2, 0], [1, 2, 3, 3, 1], schedule=s)       # diamond, repeated edge
+    _small_case(7, [0, 1, 3, 4], [1, 2, 4, 5], schedule=s)             # components + isolated
+
+
+@pytest.mark.parametrize("B", [1, 2, 31, 33, 77, 300])
+def test_ragged_batches(B):
+    r = rng(B)
+    src, dst = random_dag(r, 40, 0.1)
+    _small_case(40, src, dst, d=16, m=4, B=B, seed=B)
+
+
+@pytest.mark.parametrize("d,m", [(1, 1), (3, 2), (8, 2), (20, 5), (32, 4), (48, 8), (64, 8), (128, 6)])
+def test_widths(d, m):
+    r = rng(7)
+    src, dst = random_dag(r, 24, 0.15)
+    _small_case(24, src, dst, d=d, m=m, B=9, seed=d)
+
+
+def test_single_layer_networks_as_in_the_paper():
+    """Appendix A.7: single-layer f, g (hidden = input width)."""
+    r = rng(9)
+    src, dst = random_dag(r, 30, 0.12)
+    for sched in SCHEDULES.values():
+        _small_case(30, src, dst, d=16, m=4, B=12, layers=1, seed=3, schedule=sched)
+
+
+def test_identity_activation_and_path_counting():
+    one = net([[1.0], [1.0]], [0.0], act=1)
+    idn = net([[1.0]], [0.0], act=1)
+    w = {"d": 1, "F": 1, "m": 2, "f_down": one, "g_down": idn, "f_up": one, "g_up": idn}
+    src = np.asarray([0, 0, 1, 2], np.int32)
+    dst = np.asarray([1, 2, 3, 3], np.int32)
+    x = np.asarray([3.0, 5.0, -4.0, 11.0], np.float32).reshape(4, 1, 1)
+    g = placeto.Graph(4, src, dst)
+    Hd, Hu = placeto.placeto_embed_forward(g, placeto.Weights(w), dev_t(x))
+    assert Hd.cpu().numpy()[:, 0, 0].tolist() == [0.0, 3.0, 3.0, 7.0]
+    assert Hu.cpu().numpy()[:, 0, 0].tolist() == [23.0, 11.0, 11.0, 0.0]
+
+
+def test_max_fan_in_node():
+    n = 130
+    src = np.arange(n - 1)
+    dst = np.full(n - 1, n - 1)
+    _small_case(n, src, dst, d=32, m=4, B=20, seed=5)
+
+
+# ------------------------------------------------------ properties on GPU ---
+
+def test_deterministic_and_batch_independent():
+    cfg = configs.make("inception")
+    a = gpu_forward(cfg)
+    b = gpu_forward(cfg)
+    for k in ("H_down", "H_up", "logits", "probs"):
+        assert torch.equal(a[k], b[k]), k
+    sel = np.asarray([200, 3, 77])
+    c = gpu_forward(cfg, sel=sel)
+    for k in ("H_down", "H_up"):
+        assert_close(c[k], a[k][:, sel].cpu().numpy().astype(np.float64), k)
+    assert_close(c["logits"], a["logits"][sel].cpu().numpy().astype(np.float64), "logits")
+
+
+def test_relabelling_invariance_on_gpu():
+    cfg = configs.make("inception", normalise=True)
+    ref = gpu_forward(cfg)
+    r = rng(3)
+    n = cfg["n"]
+    perm = r.permutation(n).astype(np.int32)
+    inv = np.argsort(perm)
+    c2 = dict(cfg)
+    sh = r.permutation(len(cfg["src"]))
+    c2["src"], c2["dst"] = perm[cfg["src"]][sh], perm[cfg["dst"]][sh]
+    c2["cost"], c2["bytes"] = cfg["cost"][inv], cfg["bytes"][inv]
+    c2["dev"], c2["placed"] = cfg["dev"][:, inv], cfg["placed"][:, inv]
+    c2["cur"] = perm[cfg["cur"]]
+    out = gpu_forward(c2)
+    perm_t = torch.from_numpy(perm.astype(np.int64)).cuda()
+    assert_close(out["H_down"][perm_t], ref["H_down"].cpu().numpy().astype(np.float64), "H_down")
+    assert_close(out["logits"], ref["logits"].cpu().numpy().astype(np.float64), "logits")
+
+
+def test_schedules_agree():
+    cfg = configs.make("nmt", B=24)
+    outs = [gpu_forward(cfg, s) for s in SCHEDULES.values()]
+    ref = oracle.forward(cfg, threads=8)
+    for o in outs:
+        compare(cfg, o, ref)
+
+
+# ------------------------------------------------ fused and host variants ---
+
+def test_policy_forward_and_host_variant_match_the_separate_calls():
+    cfg = configs.make("inception")
+    ref = gpu_forward(cfg)
+    g, w = ref["graph"], ref["w"]
+    B = cfg["B"]
+    logits, probs = placeto.placeto_policy_forward(
+        g, w, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]), dev_t(cfg["cur"]),
+        dev_t(cfg["placed"]))
+    torch.cuda.synchronize()
+    assert torch.equal(logits, ref["logits"]) and torch.equal(probs, ref["probs"])
+    assert placeto.placeto_last_launch_count() >= 4
+    ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD_HOST)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_logits = torch.empty((B, cfg["m"]), dtype=torch.float32).pin_memory()
+    h_probs = torch.empty((B, cfg["m"]), dtype=torch.float32).pin_memory()
+    placeto.placeto_policy_forward_host(g, w, pin(cfg["cost"]), pin(cfg["bytes"]), pin(cfg["dev"]),
+                                        pin(cfg["cur"]), pin(cfg["placed"]), h_logits, h_probs, ws)
+    assert torch.equal(h_logits, ref["logits"].cpu()) and torch.equal(h_probs, ref["probs"].cpu())
+
+
+# ---------------------------------------------------------- error handling ---
+
+def test_argument_errors_are_reported_not_faulted():
+    cfg = configs.make("tiny")
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    B = cfg["B"]
+    X = torch.zeros((cfg["n"], B, cfg["F"]), device="cuda")
+    ws = placeto.workspace(g, w, B, placeto.CALL_EMBED)
+
+    def status(fn):
+        with pytest.raises(placeto.PlacetoError) as e:
+            fn()
+        return e.value.status
+    assert status(lambda: placeto.placeto_embed_forward(g, w, X, ws=ws[: ws.numel() // 2])) == 3
+    assert status(lambda: placeto.placeto_embed_forward(g, w, X, ws=ws, flags=3)) == 1
+    assert status(lambda: placeto.placeto_embed_forward(g, w, X, ws=ws, flags=1 << 9)) == 1
+    Xb = torch.zeros(cfg["n"] * B * cfg["F"] + 1, device="cuda")[1:].view(cfg["n"], B, cfg["F"])
+    assert status(lambda: placeto.placeto_embed_forward(g, w, Xb, ws=ws)) == 1   # misaligned
+    bad = dict(cfg["weights"]); bad["d"] = cfg["d"] + 1
+    assert status(lambda: placeto.placeto_embed_forward(g, placeto.Weights(bad), X, ws=ws)) == 1
+    # an out-of-range current node poisons that state only
+    cur = cfg["cur"].copy(); cur[3] = cfg["n"] + 5
+    Xf = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]),
+                                        dev_t(cfg["cur"]), dev_t(cfg["placed"]), cfg["m"])
+    Hd, Hu = placeto.placeto_embed_forward(g, w, Xf)
+    logits, _ = placeto.placeto_policy_logits(g, w, Xf, Hd, Hu, dev_t(cur))
+    good, _ = placeto.placeto_policy_logits(g, w, Xf, Hd, Hu, dev_t(cfg["cur"]))
+    torch.cuda.synchronize()
+    assert torch.isnan(logits[3]).all()
+    keep = [i for i in range(B) if i != 3]
+    assert torch.equal(logits[keep], good[keep])
