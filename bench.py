@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the Placeto policy forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole path (features -> two-way message passing ->
+group pooling -> head -> softmax) over one batch of synthetic placement states
+through the C ABI. The default workload is the Inception-shaped configuration
+(~300 nodes, d = 32, 256 states). Prints one JSON line.
+
+Multi-GPU (torchrun, one rank per GPU): states are independent, so every rank
+runs its own batch of the same size (weak scaling) with no data-path
+collective; the value is all ranks' states divided by the slowest rank's time.
+
+`--impl reference` times the CPU checker (oracle/) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "placement-state evaluations/sec (full-graph embed + logits)"
+UNIT = "evaluations/s"
+FP32_LANES_PER_SM = 128           # FMA lanes per SM
+L2_FLUSH_BYTES = 256 << 20        # > 126 MB L2
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="inception",
+                    help="tiny | inception | nmt | nasnet | sweepNN")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--flags", type=int, default=0, help="schedule flags of placeto.h")
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0)
+    return ap.parse_args()
+
+
+def make_workload(name: str, rank: int = 0):
+    from gen import configs, states
+    if name.startswith("sweep"):
+        cfg = configs.make_sweep(int(name[5:] or 0))
+    else:
+        cfg = configs.make(name)
+    if rank > 0:   # other ranks: same graph and weights, their own states
+        rng = np.random.Generator(np.random.PCG64(7919 * rank + 1))
+        cfg["dev"], cfg["cur"], cfg["placed"] = states.random_states(rng, cfg["n"], cfg["m"], cfg["B"])
+    return cfg
+
+
+def workload_config(cfg, n_gpus):
+    return {"workload": cfg["name"], "n_nodes": cfg["n"], "n_edges": int(len(set(zip(cfg["src"].tolist(), cfg["dst"].tolist())))),
+            "depth": cfg["depth"], "d": cfg["d"], "F": cfg["F"], "m": cfg["m"],
+            "states_per_gpu": cfg["B"], "global_states": cfg["B"] * n_gpus,
+            "parallelism": "state batch replicated per GPU, no collective" if n_gpus > 1 else "single GPU",
+            "l2": "flushed between timed steps (256 MiB memset, outside the timed events)"}
+
+
+def flops_embed(cfg):
+    d, F = cfg["d"], cfg["F"]
+    return 2.0 * (8 * d * d + 2 * d * F) * cfg["n"] * cfg["B"]
+
+
+def flops_pool(cfg):
+    d, F = cfg["d"], cfg["F"]
+    return 2.0 * (2 * d * d + d * F) * cfg["n"] * cfg["B"]
+
+
+# ------------------------------------------------------------ CPU checker ---
+
+def time_oracle(cfg, budget_s: float, threads: int):
+    """Runs the CPU checker's whole path on `cfg` repeatedly for about
+    budget_s seconds; returns (evaluations/s, seconds per pass, passes)."""
+    from oracle import oracle
+    oracle.build()
+    oracle.forward(cfg, threads=threads, states=np.arange(min(4, cfg["B"])))   # load + warm
+    t0 = time.perf_counter()
+    passes = 0
+    while True:
+        oracle.forward(cfg, threads=threads)
+        passes += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or passes >= 50:
+            break
+    return cfg["B"] * passes / el, el / passes, passes
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg = make_workload(args.workload)
+    cores = len(os.sched_getaffinity(0))
+    from oracle import oracle
+    oracle.build()
+    steps, warmup = max(1, min(args.steps, 20)), max(1, min(args.warmup, 2))
+    sample = cfg
+    # bound the work per step to roughly a second
+    est = 1e-9 * (flops_embed(cfg) + flops_pool(cfg)) / max(cores, 1) * 2.0
+    sample_desc = "full batch of %d states per step" % cfg["B"]
+    states_sel = None
+    if est > 2.0:
+        keep = max(cores, int(cfg["B"] * 2.0 / est))
+        states_sel = np.arange(min(keep, cfg["B"]))
+        sample_desc = "first %d of %d states per step" % (len(states_sel), cfg["B"])
+    nstates = cfg["B"] if states_sel is None else len(states_sel)
+    for _ in range(warmup):
+        oracle.forward(sample, threads=cores, states=states_sel)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.forward(sample, threads=cores, states=states_sel)
+    el = time.perf_counter() - t0
+    value = nstates * steps / el
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": 1e3 * el / steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(cfg, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample_desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------- clocks ----
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while running."""
+
+    def __init__(self, index: int, uuid: str | None = None):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ B200 ----
+
+def run_b200(args):
+    import torch
+    import paper_1906_08879_b200 as placeto
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = make_workload(args.workload, rank)
+    n, B, m, d, F = cfg["n"], cfg["B"], cfg["m"], cfg["d"], cfg["F"]
+    g = placeto.Graph(n, cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    dev_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    cost, nbytes = dev_t(cfg["cost"]), dev_t(cfg["bytes"])
+    devs, cur, placed = dev_t(cfg["dev"]), dev_t(cfg["cur"]), dev_t(cfg["placed"])
+    logits = torch.empty((B, m), dtype=torch.float32, device="cuda")
+    probs = torch.empty((B, m), dtype=torch.float32, device="cuda")
+    ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD_HOST, args.flags)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        placeto.placeto_policy_forward(g, w, cost, nbytes, devs, cur, placed, logits, probs, ws,
+                                       args.flags, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, count_launches=False):
+        """Sum of per-step CUDA-event times (ms) on the launching stream; L2 is
+        flushed before every step, outside the events."""
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        launches = 0
+        for i in range(steps):
+            flush.zero_()
+            starts[i].record(stream)
+            fn()
+            ends[i].record(stream)
+            if count_launches:
+                launches += placeto.placeto_last_launch_count()
+        torch.cuda.synchronize()
+        return sum(s.elapsed_time(e) for s, e in zip(starts, ends)), launches
+
+    warmup = max(args.warmup, 3)
+    sampler = ClockSampler(local, str(getattr(torch.cuda.get_device_properties(local), "uuid", "")))
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler.start()
+    total_ms, launches = timed(step, args.steps, count_launches=True)
+    barrier()
+    clocks = sampler.stop()
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    value = B * world * args.steps / (total_ms * 1e-3)
+
+    # end to end through the host-buffer entry point: pinned inputs -> device -> results on host
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_in = [pin(cfg[k]) for k in ("cost", "bytes", "dev", "cur", "placed")]
+    h_logits = torch.empty((B, m), dtype=torch.float32).pin_memory()
+    h_probs = torch.empty((B, m), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        placeto.placeto_policy_forward_host(g, w, *h_in, h_logits, h_probs, ws, args.flags, stream)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e2e_ms, _ = timed(e2e_step, args.steps)
+    barrier()
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = B * world * args.steps / (float(t.item()) * 1e-3)
+    h2d = sum(x.numel() * x.element_size() for x in h_in)
+    d2h = h_logits.numel() * 4 + h_probs.numel() * 4
+    assert torch.equal(h_logits.cuda(), logits), "host and device entry points disagree"
+
+    # the dominant kernel alone: the message-passing launch(es) of embed_forward
+    X = placeto.placeto_build_features(g, cost, nbytes, devs, cur, placed, m)
+    Hd = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
+    Hu = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
+
+    def embed_only():
+        placeto.placeto_embed_forward(g, w, X, Hd, Hu, ws, args.flags, stream)
+
+    def pool_only():
+        placeto.placeto_policy_logits(g, w, X, Hd, Hu, cur, logits, probs, ws, args.flags, stream)
+
+    for _ in range(3):
+        embed_only(); pool_only()
+    ksteps = min(args.steps, 100)
+    embed_ms, _ = timed(embed_only, ksteps)
+    embed_launches = placeto.placeto_last_launch_count()
+    pool_ms, _ = timed(pool_only, ksteps)
+    embed_ms /= ksteps
+    pool_ms /= ksteps
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    sm_count = torch.cuda.get_device_properties(0).multi_processor_count
+    sm_max_mhz = clocks["sm_max_mhz"] or 1965
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        sm_max_mhz = json.load(open(peaks_path)).get("sm_max_mhz", sm_max_mhz)
+    peak_tflops = sm_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
+    achieved = flops_embed(cfg) / (embed_ms * 1e-3) / 1e12
+    roofline = {"bound": "alu", "kernel": "message passing (embed_forward, %d launch(es))" % embed_launches,
+                "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved / peak_tflops,
+                "traffic": None,
+                "peak_source": "derived: %d SMs x 128 FP32 FMA lanes x 2 flop x %.0f MHz max SM clock"
+                               % (sm_count, sm_max_mhz),
+                "ms_per_launch": embed_ms,
+                "pooling_head_ms": pool_ms,
+                "pooling_achieved_tflops": flops_pool(cfg) / (pool_ms * 1e-3) / 1e12}
+
+    cores = len(os.sched_getaffinity(0))
+    cpu_value, cpu_s, passes = time_oracle(cfg, args.cpu_baseline_seconds, cores)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg, world), "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches, "roofline": roofline,
+            "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "%d full passes over the batch of %d states (%.2f s each)"
+                                       % (passes, B, cpu_s)}}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_b200(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
