@@ -100,11 +100,17 @@ placeto_status placeto_graph_info(const placeto_graph *g, int32_t *n, int64_t *n
  *   level_ptr[n_levels+1] : positions of each level's nodes in `order`
  *   order[n]              : node ids sorted by level, ascending id inside a level
  *   nbr_ptr[n+1], nbr[]   : neighbour ids of order[p] are nbr[nbr_ptr[p] .. nbr_ptr[p+1]), ascending
+ *   n_slots, own_slot[n], nbr_slot[] : on-chip message slots. The message of order[p] is kept
+ *                           in slot own_slot[p] (-1 if no node consumes it) from its level until
+ *                           the last level that reads it; nbr_slot[e] is the slot of nbr[e].
+ *                           Slots are shared by nodes whose lifetimes do not overlap.
  *   relation[n*n]         : relation[c*n+u] = 0 u can reach c, 1 c can reach u, 2 neither, 3 u == c
  */
 typedef struct {
     int32_t n_levels;
     const int32_t *level_ptr, *order, *nbr_ptr, *nbr;
+    int32_t n_slots;
+    const int32_t *own_slot, *nbr_slot;
 } placeto_level_view;
 placeto_status placeto_graph_host_view(const placeto_graph *g, placeto_level_view *down,
                                        placeto_level_view *up, const uint8_t **relation);

@@ -53,14 +53,16 @@ class _Weights(ctypes.Structure):
 class _LevelView(ctypes.Structure):
     _fields_ = [("n_levels", ctypes.c_int32), ("level_ptr", ctypes.POINTER(ctypes.c_int32)),
                 ("order", ctypes.POINTER(ctypes.c_int32)), ("nbr_ptr", ctypes.POINTER(ctypes.c_int32)),
-                ("nbr", ctypes.POINTER(ctypes.c_int32))]
+                ("nbr", ctypes.POINTER(ctypes.c_int32)), ("n_slots", ctypes.c_int32),
+                ("own_slot", ctypes.POINTER(ctypes.c_int32)),
+                ("nbr_slot", ctypes.POINTER(ctypes.c_int32))]
 
 
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
             "libplaceto.so is missing (%s): build it with "
-            "`python -m paper_1906_08879_b200.build`; there is no CPU fallback" % LIB_PATH)
+            "`python paper_1906_08879_b200/build.py`; there is no CPU fallback" % LIB_PATH)
     lib = ctypes.CDLL(LIB_PATH)
     lib.placeto_status_string.restype = ctypes.c_char_p
     lib.placeto_status_string.argtypes = [ctypes.c_int]
@@ -148,6 +150,10 @@ class Graph:
                 "nbr_ptr": nbr_ptr,
                 "nbr": (np.ctypeslib.as_array(v.nbr, shape=(int(nbr_ptr[-1]),)).copy()
                         if nbr_ptr[-1] > 0 else np.zeros(0, np.int32)),
+                "n_slots": v.n_slots,
+                "own_slot": np.ctypeslib.as_array(v.own_slot, shape=(n,)).copy(),
+                "nbr_slot": (np.ctypeslib.as_array(v.nbr_slot, shape=(int(nbr_ptr[-1]),)).copy()
+                             if nbr_ptr[-1] > 0 else np.zeros(0, np.int32)),
             }
         out["relation"] = np.ctypeslib.as_array(rel, shape=(n, n)).copy()
         return out

@@ -1,6 +1,7 @@
 """Builds the CUDA library in-tree with nvcc for sm_100a.
 
-``python -m paper_1906_08879_b200.build`` (or ``build()``) compiles every
+``python paper_1906_08879_b200/build.py`` (or ``build()``; run it as a script, since
+importing the package needs the library this builds) compiles every
 source under ``csrc/`` into ``libplaceto.so`` next to this file. nvcc
 cross-compiles without a GPU; the result is only usable on a B200.
 """
@@ -16,7 +17,8 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplaceto.so")
 
-SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "policy_generic.cu"]
+SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "embed_d32.cu",
+           "policy_generic.cu"]
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo",
               "-gencode", "arch=compute_100a,code=sm_100a",

@@ -141,7 +141,12 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     a.M[0] = reinterpret_cast<float *>(ws + L.msg[0]);
     a.M[1] = reinterpret_cast<float *>(ws + L.msg[1]);
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
-    return cuda_status(launch_embed_generic(a, g->info, pick_schedule(flags), stream));
+    const unsigned schedule = pick_schedule(flags);
+    if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d32_applicable(a)) {
+        cudaError_t e = launch_embed_d32(a, g->info, stream);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
+    return cuda_status(launch_embed_generic(a, g->info, schedule, stream));
 }
 
 placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const float *X,
@@ -210,13 +215,16 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
     if (cudaDeviceGetAttribute(&g->info.sm_count, cudaDevAttrMultiProcessorCount, g->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&g->info.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, g->device) != cudaSuccess)
         return fail(PLACETO_ERR_CUDA);
-    // one int allocation: per direction level_ptr, order, nbr_ptr, nbr (each padded to 4 ints)
+    // one int allocation: per direction level_ptr, order, nbr_ptr, nbr, own_slot, nbr_slot
+    // (each padded to 4 ints)
+    constexpr int kArrays = 6;
     size_t total = 0;
-    size_t offs[2][4];
+    size_t offs[2][kArrays];
     for (int dir = 0; dir < 2; ++dir) {
         const LevelPlan &p = g->host.dir[dir];
-        const size_t sizes[4] = {p.level_ptr.size(), p.order.size(), p.nbr_ptr.size(), p.nbr.size()};
-        for (int k = 0; k < 4; ++k) { offs[dir][k] = total; total += (sizes[k] + 3) & ~size_t(3); }
+        const size_t sizes[kArrays] = {p.level_ptr.size(), p.order.size(), p.nbr_ptr.size(),
+                                       p.nbr.size(), p.own_slot.size(), p.nbr_slot.size()};
+        for (int k = 0; k < kArrays; ++k) { offs[dir][k] = total; total += (sizes[k] + 3) & ~size_t(3); }
     }
     if (cudaMalloc(&g->d_ints, std::max<size_t>(total, 4) * sizeof(int)) != cudaSuccess)
         return fail(PLACETO_ERR_NO_MEMORY);
@@ -224,8 +232,9 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
         return fail(PLACETO_ERR_NO_MEMORY);
     for (int dir = 0; dir < 2; ++dir) {
         const LevelPlan &p = g->host.dir[dir];
-        const std::vector<int32_t> *vecs[4] = {&p.level_ptr, &p.order, &p.nbr_ptr, &p.nbr};
-        for (int k = 0; k < 4; ++k)
+        const std::vector<int32_t> *vecs[kArrays] = {&p.level_ptr, &p.order, &p.nbr_ptr,
+                                                     &p.nbr, &p.own_slot, &p.nbr_slot};
+        for (int k = 0; k < kArrays; ++k)
             if (!vecs[k]->empty() &&
                 cudaMemcpy(g->d_ints + offs[dir][k], vecs[k]->data(), vecs[k]->size() * sizeof(int),
                            cudaMemcpyHostToDevice) != cudaSuccess)
@@ -235,6 +244,10 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
         g->lv[dir].order = g->d_ints + offs[dir][1];
         g->lv[dir].nbr_ptr = g->d_ints + offs[dir][2];
         g->lv[dir].nbr = g->d_ints + offs[dir][3];
+        g->lv[dir].n_slots = p.n_slots;
+        g->lv[dir].own_slot = g->d_ints + offs[dir][4];
+        g->lv[dir].nbr_slot = g->d_ints + offs[dir][5];
+        g->lv[dir].n_nbr = static_cast<int>(p.nbr.size());
     }
     if (cudaMemcpy(g->d_relation, g->host.relation.data(), g->host.relation.size(),
                    cudaMemcpyHostToDevice) != cudaSuccess)
@@ -268,6 +281,9 @@ placeto_status placeto_graph_host_view(const placeto_graph *g, placeto_level_vie
         views[dir]->order = p.order.data();
         views[dir]->nbr_ptr = p.nbr_ptr.data();
         views[dir]->nbr = p.nbr.data();
+        views[dir]->n_slots = p.n_slots;
+        views[dir]->own_slot = p.own_slot.data();
+        views[dir]->nbr_slot = p.nbr_slot.data();
     }
     if (relation) *relation = g->host.relation.data();
     return PLACETO_OK;

@@ -14,6 +14,9 @@ namespace placeto {
 struct DevLevels {
     int n_levels;
     const int *level_ptr, *order, *nbr_ptr, *nbr;
+    int n_slots;                     // on-chip message slots (see plan.h)
+    const int *own_slot, *nbr_slot;
+    int n_nbr;                       // total neighbour entries
 };
 
 // One feed-forward network with device pointers.
@@ -78,6 +81,12 @@ cudaError_t launch_features(int n, int B, int m, const float *cost, const float 
 // PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.
 cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,
                                  cudaStream_t stream);
+
+// embed_d32.cu: specialised message passing for d = 32 with two-layer ReLU
+// networks of hidden width 32; returns cudaErrorNotSupported when the shapes or
+// the shared-memory budget do not fit (the caller then uses the generic kernel).
+bool embed_d32_applicable(const EmbedArgs &a);
+cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);

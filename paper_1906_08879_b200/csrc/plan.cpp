@@ -52,6 +52,37 @@ void bucket(int32_t n, const std::vector<int32_t> &level,
     }
 }
 
+// Greedy slot assignment in level order. A slot freed by a node whose last
+// consumer sits in level l can be taken again from level l + 1 on (all rows of
+// a level may run concurrently, so a slot is never reused inside the level that
+// still reads it).
+void assign_slots(int32_t n, const std::vector<int32_t> &level, LevelPlan &out) {
+    std::vector<int32_t> last_use(n, -1);
+    for (int32_t p = 0; p < n; ++p)
+        for (int32_t e = out.nbr_ptr[p]; e < out.nbr_ptr[p + 1]; ++e)
+            last_use[out.nbr[e]] = std::max(last_use[out.nbr[e]], level[out.order[p]]);
+    std::vector<std::vector<int32_t>> release(out.n_levels + 1);   // slots free from this level on
+    std::vector<int32_t> free_slots, slot_of(n, -1);
+    int32_t n_slots = 0;
+    out.own_slot.assign(n, -1);
+    for (int32_t l = 0; l < out.n_levels; ++l) {
+        for (int32_t s : release[l]) free_slots.push_back(s);
+        for (int32_t p = out.level_ptr[l]; p < out.level_ptr[l + 1]; ++p) {
+            const int32_t v = out.order[p];
+            if (last_use[v] < 0) continue;
+            int32_t s;
+            if (!free_slots.empty()) { s = free_slots.back(); free_slots.pop_back(); }
+            else s = n_slots++;
+            slot_of[v] = s;
+            out.own_slot[p] = s;
+            release[last_use[v] + 1].push_back(s);
+        }
+    }
+    out.n_slots = n_slots;
+    out.nbr_slot.resize(out.nbr.size());
+    for (size_t e = 0; e < out.nbr.size(); ++e) out.nbr_slot[e] = slot_of[out.nbr[e]];
+}
+
 }  // namespace
 
 placeto_status build_plan(int32_t n, int64_t n_edges, const int32_t *src, const int32_t *dst,
@@ -84,6 +115,8 @@ placeto_status build_plan(int32_t n, int64_t n_edges, const int32_t *src, const 
         plan.max_degree = max_degree;
         bucket(n, level_down, par, plan.dir[0]);
         bucket(n, level_up, chi, plan.dir[1]);
+        assign_slots(n, level_down, plan.dir[0]);
+        assign_slots(n, level_up, plan.dir[1]);
         plan.max_level_width = 0;
         for (int dir = 0; dir < 2; ++dir)
             for (int32_t l = 0; l < plan.dir[dir].n_levels; ++l)

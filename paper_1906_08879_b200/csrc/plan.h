@@ -15,6 +15,13 @@ struct LevelPlan {
     std::vector<int32_t> order;      // [n] node ids by level, ascending id inside a level
     std::vector<int32_t> nbr_ptr;    // [n + 1] by position in order
     std::vector<int32_t> nbr;        // neighbour ids (parents for down, children for up)
+    // On-chip message slots. A node's message f([h || x]) is live from its own
+    // level until the last level that consumes it; nodes whose lifetimes do not
+    // overlap share a slot, so a block can keep all live messages of its states
+    // in shared memory instead of n rows in global memory.
+    int32_t n_slots = 0;
+    std::vector<int32_t> own_slot;   // [n] by position: slot the node writes, -1 if nobody reads it
+    std::vector<int32_t> nbr_slot;   // [nbr.size()] slot of each neighbour
 };
 
 struct HostPlan {

@@ -27,7 +27,8 @@ pytestmark = pytest.mark.gpu
 
 TOL_ELEM, TOL_NORM = 1e-4, 2e-5
 SCHEDULES = {"sliced": placeto.PLACETO_SLICED, "per_level": placeto.PLACETO_PER_LEVEL,
-             "cooperative": placeto.PLACETO_COOPERATIVE}
+             "cooperative": placeto.PLACETO_COOPERATIVE,
+             "generic_sliced": placeto.PLACETO_SLICED | placeto.PLACETO_GENERIC}
 
 
 def dev_t(a):

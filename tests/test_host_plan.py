@@ -56,6 +56,8 @@ def _check_plan(n, src, dst):
             # longest-path layering: one more than the deepest neighbour
             want = 1 + max(level[u] for u in nbrs[node]) if nbrs[node] else 0
             assert level[node] == want
+    for name in ("down", "up"):
+        _check_slots(view[name])
     assert info["n_levels_down"] == view["down"]["n_levels"] == graphs.depth(n, src, dst)
     assert info["n_levels_up"] == view["up"]["n_levels"] == info["n_levels_down"]
     R = closure(n, src, dst)
@@ -66,6 +68,34 @@ def _check_plan(n, src, dst):
     np.fill_diagonal(want, 3)
     np.testing.assert_array_equal(rel, want)
     g.close()
+
+
+def _check_slots(v):
+    """Replays the level walk: every neighbour's slot must still hold that
+    neighbour's message when it is read, and a level never writes a slot that
+    the same level reads."""
+    n = len(v["order"])
+    holder = {}                                   # slot -> node whose message it holds
+    consumers = np.zeros(n, dtype=bool)
+    consumers[v["nbr"]] = True
+    for l in range(v["n_levels"]):
+        span = range(v["level_ptr"][l], v["level_ptr"][l + 1])
+        read = set()
+        for p in span:
+            for e in range(v["nbr_ptr"][p], v["nbr_ptr"][p + 1]):
+                s = v["nbr_slot"][e]
+                assert 0 <= s < v["n_slots"] and holder[s] == v["nbr"][e]
+                read.add(s)
+        written = set()
+        for p in span:
+            s = v["own_slot"][p]
+            node = v["order"][p]
+            assert (s >= 0) == bool(consumers[node])
+            if s >= 0:
+                assert s < v["n_slots"] and s not in read and s not in written
+                written.add(s)
+                holder[s] = node
+    assert v["n_slots"] <= max(1, int(consumers.sum()))
 
 
 def test_plan_small_shapes():
