@@ -74,7 +74,8 @@ placeto_status pool_weights_ok(const placeto_weights *w) {
 
 struct Layout {
     size_t msg[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
-    int chunks, chunk_nodes;
+    int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
+    int chunks32, chunk_nodes32;   // and of the d = 32 kernel (0 when it cannot apply)
 };
 
 // Workspace layout shared by every call; a call uses the leading part it needs.
@@ -90,8 +91,10 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         L.msg[0] = take(n * B * d * sizeof(float));
         L.msg[1] = take(n * B * d * sizeof(float));
     }
+    if (w->d == 32 && w->F >= 4 && w->F <= 16 && (w->F & 3) == 0)
+        pool_d32_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
     if (call == PLACETO_CALL_LOGITS || call >= PLACETO_CALL_FORWARD)
-        L.partial = take((size_t)L.chunks * B * 3 * d * sizeof(float));
+        L.partial = take((size_t)std::max(L.chunks, L.chunks32) * B * 3 * d * sizeof(float));
     if (call >= PLACETO_CALL_FORWARD) {
         L.X = take(n * B * F * sizeof(float));
         L.H[0] = take(n * B * d * sizeof(float));
@@ -141,6 +144,7 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     a.M[0] = reinterpret_cast<float *>(ws + L.msg[0]);
     a.M[1] = reinterpret_cast<float *>(ws + L.msg[1]);
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
+    a.max_level_width = g->host.max_level_width;
     const unsigned schedule = pick_schedule(flags);
     if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d32_applicable(a)) {
         cudaError_t e = launch_embed_d32(a, g->info, stream);
@@ -153,7 +157,6 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
                         const float *H_down, const float *H_up, const int32_t *cur, int B,
                         float *logits, float *probs, char *ws, const Layout &L, uint32_t flags,
                         cudaStream_t stream) {
-    (void)flags;
     PoolArgs a;
     for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
     a.head = to_dev(w->head);
@@ -163,6 +166,12 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     a.partial = reinterpret_cast<float *>(ws + L.partial);
     a.logits = logits; a.probs = probs;
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d; a.m = w->m;
+    if (!(flags & PLACETO_GENERIC) && L.chunks32 > 0 && pool_d32_applicable(a)) {
+        a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
+        cudaError_t e = launch_pool_d32(a, g->info, stream);
+        if (e == cudaSuccess) return cuda_status(launch_pool_head(a, stream));
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     a.chunks = L.chunks; a.chunk_nodes = L.chunk_nodes;
     return cuda_status(launch_policy_generic(a, g->info, stream));
 }

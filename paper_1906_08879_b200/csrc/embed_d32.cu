@@ -13,7 +13,12 @@
 //   - Messages never leave the SM: m_u lives in a shared-memory slot from the
 //     level of u until its last consumer's level (slots assigned on the host).
 //     Global traffic is the compulsory part only: read x, write h.
-//   - The level schedule (order, CSR, slots) is staged in shared memory.
+//   - The level schedule (order, CSR, slots) is staged in shared memory, and the
+//     raw features of the next level are copied asynchronously (cp.async) into a
+//     double-buffered staging area while the current level computes, so no DRAM
+//     latency sits on the level-to-level critical path.
+#include <cuda_pipeline.h>
+
 #include <algorithm>
 
 #include "kernels.cuh"
@@ -30,29 +35,103 @@ struct D32Plan {
     int S;          // states per slice
     int n_slices;
     int ints_in_smem;
+    int x_floats;   // floats of one feature staging buffer (widest level x S x F, padded)
     size_t smem_bytes;
 };
 
-// o0/o1 = bias + in0/in1 . w  over K inputs read as broadcast float4 from shared memory.
-template <int K>
-__device__ __forceinline__ void matvec2(const float (&w)[K], float bias, const float *in0,
-                                        const float *in1, float &o0, float &o1) {
-    float a0 = bias, a1 = 0.f, b0 = bias, b1 = 0.f;
+// out[r] = bias + in[r] . w for R rows whose K inputs are read as broadcast
+// float4 from shared memory; 4 / R independent accumulators per row keep the
+// FMA pipe busy without lengthening the dependent chain.
+template <int R, int K>
+__device__ __forceinline__ void matvec(const float (&w)[K], float bias, const float *in,
+                                       int row_stride, float (&out)[R]) {
+    constexpr int NA = 4 / R;
+    float acc[R][NA];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int t = 0; t < NA; ++t) acc[r][t] = t == 0 ? bias : 0.f;
 #pragma unroll
     for (int k = 0; k < K; k += 4) {
-        const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
-        const float4 v = *reinterpret_cast<const float4 *>(in1 + k);
-        a0 = fmaf(u.x, w[k], a0);
-        b0 = fmaf(v.x, w[k], b0);
-        a1 = fmaf(u.y, w[k + 1], a1);
-        b1 = fmaf(v.y, w[k + 1], b1);
-        a0 = fmaf(u.z, w[k + 2], a0);
-        b0 = fmaf(v.z, w[k + 2], b0);
-        a1 = fmaf(u.w, w[k + 3], a1);
-        b1 = fmaf(v.w, w[k + 3], b1);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float4 u = *reinterpret_cast<const float4 *>(in + r * row_stride + k);
+            acc[r][0 % NA] = fmaf(u.x, w[k], acc[r][0 % NA]);
+            acc[r][1 % NA] = fmaf(u.y, w[k + 1], acc[r][1 % NA]);
+            acc[r][2 % NA] = fmaf(u.z, w[k + 2], acc[r][2 % NA]);
+            acc[r][3 % NA] = fmaf(u.w, w[k + 3], acc[r][3 % NA]);
+        }
     }
-    o0 = a0 + a1;
-    o1 = b0 + b1;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        float s = acc[r][0];
+#pragma unroll
+        for (int t = 1; t < NA; ++t) s += acc[r][t];
+        out[r] = s;
+    }
+}
+
+struct Weights32 {
+    float g1[kD], g2[kD], f2[kD];
+    float bg1, bg2, bf1, bf2;
+};
+
+// Carries R rows of one level through gather -> g -> store h -> f -> store m.
+// A, Bf: the warp's two exchange buffers, R rows of KF floats each.
+template <int R, int KF>
+__device__ __forceinline__ void run_rows(const Weights32 &w, const float (&wf1)[KF], int first_row,
+                                         int n_rows, int p0, int nb, int S, int F, int lane,
+                                         const int *order, const int *nbr_ptr, const int *nbr_slot,
+                                         const int *own_slot, float *msg, const float *xs,
+                                         float *__restrict__ H, size_t B, int b_first, float *A,
+                                         float *Bf) {
+    int pos[R], st[R];
+    bool live[R];
+    float x[R], acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        live[r] = first_row + r < n_rows;
+        const int row = live[r] ? first_row + r : first_row;      // a missing row repeats the first
+        const int q = row / nb;
+        st[r] = row - q * nb;
+        pos[r] = p0 + q;
+        x[r] = lane < F ? xs[row * F + lane] : 0.f;
+        float g = 0.f;
+        for (int e = nbr_ptr[pos[r]]; e < nbr_ptr[pos[r] + 1]; ++e)
+            g += msg[((size_t)nbr_slot[e] * S + st[r]) * kD + lane];
+        A[r * KF + lane] = g;
+    }
+    __syncwarp();
+    matvec<R, kD>(w.g1, w.bg1, A, KF, acc);
+#pragma unroll
+    for (int r = 0; r < R; ++r) Bf[r * KF + lane] = fmaxf(acc[r], 0.f);
+    __syncwarp();
+    matvec<R, kD>(w.g2, w.bg2, Bf, KF, acc);
+    bool any = false;
+    int slot[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        acc[r] = fmaxf(acc[r], 0.f);
+        if (live[r]) H[((size_t)order[pos[r]] * B + b_first + st[r]) * kD + lane] = acc[r];
+        slot[r] = own_slot[pos[r]];
+        any |= slot[r] >= 0;
+    }
+    if (!any) return;                       // nobody consumes these messages (warp-uniform)
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        A[r * KF + lane] = acc[r];
+        if (lane < KF - kD) A[r * KF + kD + lane] = x[r];
+    }
+    __syncwarp();
+    matvec<R, KF>(wf1, w.bf1, A, KF, acc);
+#pragma unroll
+    for (int r = 0; r < R; ++r) Bf[r * KF + lane] = fmaxf(acc[r], 0.f);
+    __syncwarp();
+    matvec<R, kD>(w.f2, w.bf2, Bf, KF, acc);
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+        if (live[r] && slot[r] >= 0)
+            msg[((size_t)slot[r] * S + st[r]) * kD + lane] = fmaxf(acc[r], 0.f);
 }
 
 template <int F4>   // feature width padded to 4 * F4
@@ -67,7 +146,7 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     const int b_first = blockIdx.x * p.S;
     const int nb = min(p.S, B - b_first);
 
-    // ---- shared memory: [schedule ints][message slots][per-warp exchange buffers]
+    // ---- shared memory: [schedule ints][message slots][feature staging x2][exchange buffers]
     const int *level_ptr = lv.level_ptr, *order = lv.order, *nbr_ptr = lv.nbr_ptr;
     const int *nbr_slot = lv.nbr_slot, *own_slot = lv.own_slot;
     float *fsm = smem;
@@ -87,69 +166,68 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         fsm = reinterpret_cast<float *>(ism);
     }
     float *msg = fsm;                                       // [n_slots][S][32]
-    float *xbuf = msg + (size_t)lv.n_slots * p.S * kD + (size_t)warp * 4 * KF;
-    float *A0 = xbuf, *A1 = xbuf + KF, *B0 = xbuf + 2 * KF, *B1 = xbuf + 3 * KF;
+    float *xstage = msg + (size_t)lv.n_slots * p.S * kD;    // [2][x_floats]
+    float *xbuf = xstage + 2 * (size_t)p.x_floats + (size_t)warp * 4 * KF;
+    float *A = xbuf, *Bf = xbuf + 2 * KF;
 
     // ---- this lane's weight columns
     const DevMlp f = a.f[dir], g = a.g[dir];
-    float wg1[kD], wg2[kD], wf1[KF], wf2[kD];
+    Weights32 w;
+    float wf1[KF];
 #pragma unroll
     for (int k = 0; k < kD; ++k) {
-        wg1[k] = g.W1[k * kD + lane];
-        wg2[k] = g.W2[k * kD + lane];
-        wf2[k] = f.W2[k * kD + lane];
+        w.g1[k] = g.W1[k * kD + lane];
+        w.g2[k] = g.W2[k * kD + lane];
+        w.f2[k] = f.W2[k * kD + lane];
     }
 #pragma unroll
     for (int k = 0; k < KF; ++k) wf1[k] = (k < kD + F) ? f.W1[k * kD + lane] : 0.f;
-    const float bg1 = g.b1[lane], bg2 = g.b2[lane], bf1 = f.b1[lane], bf2 = f.b2[lane];
+    w.bg1 = g.b1[lane]; w.bg2 = g.b2[lane]; w.bf1 = f.b1[lane]; w.bf2 = f.b2[lane];
     const float *__restrict__ X = a.X;
     float *__restrict__ H = a.H[dir];
     __syncthreads();
 
-    for (int level = 0; level < lv.n_levels; ++level) {
-        const int p0 = level_ptr[level];
-        const int rows = (level_ptr[level + 1] - p0) * nb;
-        for (int r = 2 * warp; r < rows; r += 2 * kWarps) {
-            // rows r and r + 1 (the second may not exist: it then repeats the first)
-            const bool two = r + 1 < rows;
-            const int q0 = r / nb, s0 = r - q0 * nb;
-            const int r1 = two ? r + 1 : r;
-            const int q1 = r1 / nb, s1 = r1 - q1 * nb;
-            const int pos0 = p0 + q0, pos1 = p0 + q1;
-            const int v0 = order[pos0], v1 = order[pos1];
-            const size_t row0 = (size_t)v0 * B + b_first + s0, row1 = (size_t)v1 * B + b_first + s1;
-            // raw features, needed at the third layer: issue the loads first
-            float x0 = 0.f, x1 = 0.f;
-            if (lane < F) { x0 = X[row0 * F + lane]; x1 = X[row1 * F + lane]; }
-            // gather: sum of the neighbours' messages (column `lane`)
-            float g0 = 0.f, g1 = 0.f;
-            for (int e = nbr_ptr[pos0]; e < nbr_ptr[pos0 + 1]; ++e)
-                g0 += msg[((size_t)nbr_slot[e] * p.S + s0) * kD + lane];
-            for (int e = nbr_ptr[pos1]; e < nbr_ptr[pos1 + 1]; ++e)
-                g1 += msg[((size_t)nbr_slot[e] * p.S + s1) * kD + lane];
-            A0[lane] = g0; A1[lane] = g1;
-            __syncwarp();
-            float t0, t1;
-            matvec2<kD>(wg1, bg1, A0, A1, t0, t1);
-            B0[lane] = fmaxf(t0, 0.f); B1[lane] = fmaxf(t1, 0.f);
-            __syncwarp();
-            matvec2<kD>(wg2, bg2, B0, B1, t0, t1);
-            t0 = fmaxf(t0, 0.f); t1 = fmaxf(t1, 0.f);
-            H[row0 * kD + lane] = t0;
-            if (two) H[row1 * kD + lane] = t1;
-            const int slot0 = own_slot[pos0], slot1 = own_slot[pos1];
-            if (slot0 >= 0 || slot1 >= 0) {          // somebody consumes the message
-                A0[lane] = t0; A1[lane] = t1;
-                if (lane < 4 * F4) { A0[kD + lane] = x0; A1[kD + lane] = x1; }
-                __syncwarp();
-                matvec2<KF>(wf1, bf1, A0, A1, t0, t1);
-                B0[lane] = fmaxf(t0, 0.f); B1[lane] = fmaxf(t1, 0.f);
-                __syncwarp();
-                matvec2<kD>(wf2, bf2, B0, B1, t0, t1);
-                if (slot0 >= 0) msg[((size_t)slot0 * p.S + s0) * kD + lane] = fmaxf(t0, 0.f);
-                if (two && slot1 >= 0) msg[((size_t)slot1 * p.S + s1) * kD + lane] = fmaxf(t1, 0.f);
+    // Asynchronous copy of one level's raw features (rows of the slice) into a
+    // staging buffer, so that the next level's x is on chip when it is needed.
+    const int per_node = nb * F;             // floats per node, contiguous in X
+    auto prefetch = [&](int level) {
+        const int q0 = level_ptr[level], width = level_ptr[level + 1] - q0;
+        float *dst = xstage + (size_t)(level & 1) * p.x_floats;
+        if ((F & 3) == 0) {
+            const int per = per_node >> 2;
+            for (int i = threadIdx.x; i < width * per; i += kThreads) {
+                const int q = i / per, off = (i - q * per) * 4;
+                __pipeline_memcpy_async(dst + q * per_node + off,
+                                        X + ((size_t)order[q0 + q] * B + b_first) * F + off, 16);
+            }
+        } else {
+            for (int i = threadIdx.x; i < width * per_node; i += kThreads) {
+                const int q = i / per_node, off = i - q * per_node;
+                __pipeline_memcpy_async(dst + i, X + ((size_t)order[q0 + q] * B + b_first) * F + off, 4);
             }
         }
+        __pipeline_commit();
+    };
+    prefetch(0);
+    __pipeline_wait_prior(0);
+    __syncthreads();
+
+    for (int level = 0; level < lv.n_levels; ++level) {
+        if (level + 1 < lv.n_levels) prefetch(level + 1);
+        const int p0 = level_ptr[level];
+        const int rows = (level_ptr[level + 1] - p0) * nb;
+        const float *xs = xstage + (size_t)(level & 1) * p.x_floats;
+        if (rows <= kWarps) {
+            // narrow level: one row per warp, shortest dependent chains
+            if (warp < rows)
+                run_rows<1, KF>(w, wf1, warp, rows, p0, nb, p.S, F, lane, order, nbr_ptr, nbr_slot,
+                                own_slot, msg, xs, H, B, b_first, A, Bf);
+        } else {
+            for (int r = 2 * warp; r < rows; r += 2 * kWarps)
+                run_rows<2, KF>(w, wf1, r, rows, p0, nb, p.S, F, lane, order, nbr_ptr, nbr_slot,
+                                own_slot, msg, xs, H, B, b_first, A, Bf);
+        }
+        __pipeline_wait_prior(0);
         __syncthreads();
     }
 }
@@ -185,8 +263,10 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
         ints = std::max(ints, s);
     }
     const size_t xbuf = (size_t)kWarps * 4 * KF * sizeof(float);
+    auto x_floats = [&](int S) { return (a.max_level_width * S * a.F + 3) & ~3; };
     auto need = [&](int S, bool with_ints) {
-        return (size_t)max_slots * S * kD * sizeof(float) + xbuf + (with_ints ? ints * sizeof(int) : 0);
+        return (size_t)max_slots * S * kD * sizeof(float) + 2 * (size_t)x_floats(S) * sizeof(float) +
+               xbuf + (with_ints ? ints * sizeof(int) : 0);
     };
     p.ints_in_smem = 1;
     if (need(p.S, true) > budget) {
@@ -199,6 +279,7 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
         }
     }
     p.n_slices = (a.B + p.S - 1) / p.S;
+    p.x_floats = x_floats(p.S);
     p.smem_bytes = need(p.S, p.ints_in_smem != 0);
     void (*kern)(const EmbedArgs, const D32Plan) = nullptr;
     switch (F4) {

@@ -51,6 +51,7 @@ struct EmbedArgs {
     float *H[2];   // outputs [n][B][d]
     float *M[2];   // messages f([h || x]) per node and state, [n][B][d] (workspace)
     int n, B, F, d;
+    int max_level_width;   // widest level over both directions
 };
 
 struct PoolArgs {
@@ -91,5 +92,12 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);
 cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
+// adds the chunk partial sums, applies h_i, the head and the softmax (one block per state)
+cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream);
+
+// policy_d32.cu: specialised partial sums for d = 32, F a multiple of 4, single-layer ReLU l_i
+bool pool_d32_applicable(const PoolArgs &a);
+void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
+cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
 }  // namespace placeto

@@ -1,0 +1,197 @@
+// Step 3 of the policy (Sec. 2.2 step 3 of the Placeto paper) specialised for
+// d = 32 with single-layer ReLU l_i: the per-set sums
+//   sum_{u in S_i(c)} l_i(e_u),   e_u = [h_down_u || h_up_u || x_u],
+// for a chunk of nodes and a tile of 16 states per block, written as partial
+// sums that the head kernel adds up in chunk order.
+//
+// A block first copies its whole tile (chunk x 16 states of H_down, H_up, X) and
+// the three weight matrices into shared memory with cp.async. Warp w owns state
+// w of the tile. For each set i in turn it loads column `lane` of W_i into
+// registers, scans the relation row of its state's current node over the chunk
+// (ballot), and pushes the rows of set i through the 32 x (64 + F) product two at
+// a time, reading the inputs as broadcast 128-bit shared loads; the sums stay in
+// registers. Summation order is ascending node id: deterministic.
+#include <cuda_pipeline.h>
+
+#include <algorithm>
+
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kD = 32;
+constexpr int kWarps = 16;             // = states per block
+constexpr int kThreads = kWarps * 32;
+
+struct Pool32Plan {
+    int chunk_nodes, chunks;
+    size_t smem_bytes;
+};
+
+template <int R, int K>
+__device__ __forceinline__ void fma_rows(const float *w, const float *const (&in)[R],
+                                         float (&acc)[R][2]) {
+#pragma unroll
+    for (int k = 0; k < K; k += 4) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float4 u = *reinterpret_cast<const float4 *>(in[r] + k);
+            acc[r][0] = fmaf(u.x, w[k], acc[r][0]);
+            acc[r][1] = fmaf(u.y, w[k + 1], acc[r][1]);
+            acc[r][0] = fmaf(u.z, w[k + 2], acc[r][0]);
+            acc[r][1] = fmaf(u.w, w[k + 3], acc[r][1]);
+        }
+    }
+}
+
+template <int F4>
+__global__ void __launch_bounds__(kThreads, 1)
+pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
+    constexpr int FP = 4 * F4;             // padded feature width
+    constexpr int E = 2 * kD + FP;
+    extern __shared__ __align__(16) float smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = a.n, B = a.B, F = a.F;
+    const int chunk = blockIdx.x;
+    const int u0 = chunk * p.chunk_nodes, nu = min(n, u0 + p.chunk_nodes) - u0;
+    const int b0 = blockIdx.y * kWarps, nb = min(kWarps, B - b0);
+
+    float *Ws = smem;                                   // [3][E][32], rows past 64 + F are zero
+    float *bs = Ws + 3 * E * kD;                        // [3][32]
+    float *hd = bs + 3 * kD;                            // [chunk][16][32]
+    float *hu = hd + (size_t)p.chunk_nodes * kWarps * kD;
+    float *xs = hu + (size_t)p.chunk_nodes * kWarps * kD;   // [chunk][16][FP]
+
+    // ---- stage weights and the tile
+    for (int i = 0; i < 3; ++i) {
+        const float *W = a.l[i].W1;
+        for (int t = threadIdx.x; t < E * kD / 4; t += kThreads) {
+            const int k = (t * 4) / kD;
+            if (k < 2 * kD + F) __pipeline_memcpy_async(Ws + i * E * kD + t * 4, W + t * 4, 16);
+            else *reinterpret_cast<float4 *>(Ws + i * E * kD + t * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (threadIdx.x < kD) bs[i * kD + threadIdx.x] = a.l[i].b1[threadIdx.x];
+    }
+    {
+        const int per_h = nb * kD / 4;                  // 16-byte pieces per node
+        for (int t = threadIdx.x; t < nu * per_h; t += kThreads) {
+            const int q = t / per_h, off = (t - q * per_h) * 4;
+            const size_t src = ((size_t)(u0 + q) * B + b0) * kD + off;
+            __pipeline_memcpy_async(hd + (size_t)q * kWarps * kD + off, a.H[0] + src, 16);
+            __pipeline_memcpy_async(hu + (size_t)q * kWarps * kD + off, a.H[1] + src, 16);
+        }
+        const int per_x = nb * F / 4;                   // F is a multiple of 4 here, FP == F
+        for (int t = threadIdx.x; t < nu * per_x; t += kThreads) {
+            const int q = t / per_x, off = (t - q * per_x) * 4;
+            __pipeline_memcpy_async(xs + (size_t)q * kWarps * FP + off,
+                                    a.X + ((size_t)(u0 + q) * B + b0) * F + off, 16);
+        }
+    }
+    __pipeline_commit();
+    __pipeline_wait_prior(0);
+    __syncthreads();
+
+    if (warp >= nb) return;
+    const int b = b0 + warp;
+    const int c = a.cur[b];
+    const bool valid = c >= 0 && c < n;
+    const uint8_t *rel = a.relation + (size_t)(valid ? c : 0) * n + u0;
+    float *out = a.partial + ((size_t)chunk * B + b) * 3 * kD;
+    for (int i = 0; i < 3; ++i) {
+        float w[E];
+#pragma unroll
+        for (int k = 0; k < E; ++k) w[k] = Ws[(i * E + k) * kD + lane];
+        const float bias = bs[i * kD + lane];
+        float total = 0.f;
+        for (int base = 0; base < nu && valid; base += 32) {
+            const int q = base + lane;
+            unsigned mask = __ballot_sync(0xffffffffu, q < nu && rel[q] == i);
+            while (mask) {
+                const int qa = base + __ffs(mask) - 1;
+                mask &= mask - 1;
+                if (mask) {
+                    const int qb = base + __ffs(mask) - 1;
+                    mask &= mask - 1;
+                    float acc[2][2] = {{bias, 0.f}, {bias, 0.f}};
+                    const size_t ra = (size_t)qa * kWarps + warp, rb = (size_t)qb * kWarps + warp;
+                    const float *const pd[2] = {hd + ra * kD, hd + rb * kD};
+                    const float *const pu[2] = {hu + ra * kD, hu + rb * kD};
+                    const float *const px[2] = {xs + ra * FP, xs + rb * FP};
+                    fma_rows<2, kD>(w, pd, acc);
+                    fma_rows<2, kD>(w + kD, pu, acc);
+                    fma_rows<2, FP>(w + 2 * kD, px, acc);
+                    total += fmaxf(acc[0][0] + acc[0][1], 0.f);
+                    total += fmaxf(acc[1][0] + acc[1][1], 0.f);
+                } else {
+                    float acc[1][2] = {{bias, 0.f}};
+                    const size_t ra = (size_t)qa * kWarps + warp;
+                    const float *const pd[1] = {hd + ra * kD};
+                    const float *const pu[1] = {hu + ra * kD};
+                    const float *const px[1] = {xs + ra * FP};
+                    fma_rows<1, kD>(w, pd, acc);
+                    fma_rows<1, kD>(w + kD, pu, acc);
+                    fma_rows<1, FP>(w + 2 * kD, px, acc);
+                    total += fmaxf(acc[0][0] + acc[0][1], 0.f);
+                }
+            }
+        }
+        out[i * kD + lane] = total;
+    }
+}
+
+bool relu1(const DevMlp &m, int in) {
+    return m.n_layers == 1 && m.in_dim == in && m.out_dim == kD && m.act == 0 && m.final_act == 1;
+}
+
+}  // namespace
+
+bool pool_d32_applicable(const PoolArgs &a) {
+    if (a.d != kD || a.F < 4 || a.F > 16 || (a.F & 3)) return false;
+    for (int i = 0; i < 3; ++i)
+        if (!relu1(a.l[i], 2 * kD + a.F)) return false;
+    return true;
+}
+
+// Nodes per chunk and number of chunks for a batch of B states.
+void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks) {
+    const int E = 2 * kD + F;
+    const size_t budget = (size_t)std::min(di.max_smem_optin, 227 * 1024) - 1024;
+    const size_t fixed = (size_t)(3 * E * kD + 3 * kD) * sizeof(float);
+    const size_t per_node = (size_t)kWarps * E * sizeof(float);
+    const int cap = std::max(1, (int)((budget - fixed) / per_node));
+    const int tiles = (B + kWarps - 1) / kWarps;
+    int c = (n + cap - 1) / cap;
+    // a single wave: give every SM a block if the chunks can be made smaller
+    if (c * tiles < di.sm_count) c = std::max(c, std::min(di.sm_count / tiles, (n + 7) / 8));
+    c = std::max(1, c);
+    *chunk_nodes = (n + c - 1) / c;
+    *chunks = (n + *chunk_nodes - 1) / *chunk_nodes;
+}
+
+cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+    Pool32Plan p;
+    p.chunk_nodes = a.chunk_nodes;
+    p.chunks = a.chunks;
+    const int E = 2 * kD + a.F;
+    p.smem_bytes = ((size_t)(3 * E * kD + 3 * kD) + (size_t)p.chunk_nodes * kWarps * E) * sizeof(float);
+    if (p.smem_bytes > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
+    void (*kern)(const PoolArgs, const Pool32Plan) = nullptr;
+    switch (a.F / 4) {
+        case 1: kern = pool_d32_kernel<1>; break;
+        case 2: kern = pool_d32_kernel<2>; break;
+        case 3: kern = pool_d32_kernel<3>; break;
+        case 4: kern = pool_d32_kernel<4>; break;
+        default: return cudaErrorNotSupported;
+    }
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)p.smem_bytes);
+    if (err != cudaSuccess) return err;
+    dim3 grid(p.chunks, (a.B + kWarps - 1) / kWarps);
+    kern<<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace placeto

@@ -239,15 +239,19 @@ cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaS
     count_launch();
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
+    return launch_pool_head(a, stream);
+}
 
+cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
     const int Z = 5 * a.d + a.F;
     int tmp_floats = a.head.n_layers == 2 ? a.head.hidden_dim : 0;
     for (int i = 0; i < 3; ++i)
         if (a.h[i].n_layers == 2) tmp_floats = std::max(tmp_floats, a.h[i].hidden_dim);
     tmp_floats = (tmp_floats + 3) & ~3;
     const size_t head_smem = (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m + 4) * sizeof(float);
-    err = cudaFuncSetAttribute(pool_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)head_smem);
+    cudaError_t err = cudaFuncSetAttribute(pool_head_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)head_smem);
     if (err != cudaSuccess) return err;
     pool_head_kernel<<<a.B, kHeadThreads, head_smem, stream>>>(a, tmp_floats);
     count_launch();
