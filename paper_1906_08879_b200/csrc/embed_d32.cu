@@ -9,7 +9,8 @@
 //     a row (node, state) through gather -> g1 -> g2 -> f1 -> f2 on its own.
 //     Between layers the 32 outputs are exchanged through a per-warp shared
 //     buffer and read back as broadcast 128-bit loads: 4 FMAs per shared load.
-//   - Two rows are in flight per warp for instruction-level parallelism.
+//   - Two states of a node are in flight per warp (one on narrow levels), with
+//     four accumulators per row, for instruction-level parallelism.
 //   - Messages never leave the SM: m_u lives in a shared-memory slot from the
 //     level of u until its last consumer's level (slots assigned on the host).
 //     Global traffic is the compulsory part only: read x, write h.
@@ -40,35 +41,30 @@ struct D32Plan {
 };
 
 // out[r] = bias + in[r] . w for R rows whose K inputs are read as broadcast
-// float4 from shared memory; 4 / R independent accumulators per row keep the
+// float4 from shared memory; four independent accumulators per row keep the
 // FMA pipe busy without lengthening the dependent chain.
 template <int R, int K>
 __device__ __forceinline__ void matvec(const float (&w)[K], float bias, const float *in,
                                        int row_stride, float (&out)[R]) {
-    constexpr int NA = 4 / R;
-    float acc[R][NA];
+    float acc[R][4];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int t = 0; t < NA; ++t) acc[r][t] = t == 0 ? bias : 0.f;
+    for (int r = 0; r < R; ++r) {
+        acc[r][0] = bias;
+        acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+    }
 #pragma unroll
     for (int k = 0; k < K; k += 4) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             const float4 u = *reinterpret_cast<const float4 *>(in + r * row_stride + k);
-            acc[r][0 % NA] = fmaf(u.x, w[k], acc[r][0 % NA]);
-            acc[r][1 % NA] = fmaf(u.y, w[k + 1], acc[r][1 % NA]);
-            acc[r][2 % NA] = fmaf(u.z, w[k + 2], acc[r][2 % NA]);
-            acc[r][3 % NA] = fmaf(u.w, w[k + 3], acc[r][3 % NA]);
+            acc[r][0] = fmaf(u.x, w[k], acc[r][0]);
+            acc[r][1] = fmaf(u.y, w[k + 1], acc[r][1]);
+            acc[r][2] = fmaf(u.z, w[k + 2], acc[r][2]);
+            acc[r][3] = fmaf(u.w, w[k + 3], acc[r][3]);
         }
     }
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        float s = acc[r][0];
-#pragma unroll
-        for (int t = 1; t < NA; ++t) s += acc[r][t];
-        out[r] = s;
-    }
+    for (int r = 0; r < R; ++r) out[r] = (acc[r][0] + acc[r][1]) + (acc[r][2] + acc[r][3]);
 }
 
 struct Weights32 {
@@ -76,47 +72,49 @@ struct Weights32 {
     float bg1, bg2, bf1, bf2;
 };
 
-// Carries R rows of one level through gather -> g -> store h -> f -> store m.
-// A, Bf: the warp's two exchange buffers, R rows of KF floats each.
+// Carries R states (s0 .. s0 + R - 1 of the slice; the last may be missing and
+// then repeats s0) of the node at position `pos` through
+// gather -> g -> store h -> f -> store m. The R rows share the node, so the
+// schedule lookups are done once. A, Bf: the warp's exchange buffers, R rows of
+// KF floats each. All shared-memory offsets are 32-bit.
 template <int R, int KF>
-__device__ __forceinline__ void run_rows(const Weights32 &w, const float (&wf1)[KF], int first_row,
-                                         int n_rows, int p0, int nb, int S, int F, int lane,
-                                         const int *order, const int *nbr_ptr, const int *nbr_slot,
-                                         const int *own_slot, float *msg, const float *xs,
-                                         float *__restrict__ H, size_t B, int b_first, float *A,
-                                         float *Bf) {
-    int pos[R], st[R];
-    bool live[R];
+__device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[KF], int pos,
+                                         int q, int s0, bool last_live, int nb, int S, int F,
+                                         int lane, const int *order, const int *nbr_ptr,
+                                         const int *nbr_slot, const int *own_slot, float *msg,
+                                         const float *xs, float *__restrict__ H, size_t B,
+                                         int b_first, float *A, float *Bf) {
+    int st[R];
     float x[R], acc[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        live[r] = first_row + r < n_rows;
-        const int row = live[r] ? first_row + r : first_row;      // a missing row repeats the first
-        const int q = row / nb;
-        st[r] = row - q * nb;
-        pos[r] = p0 + q;
-        x[r] = lane < F ? xs[row * F + lane] : 0.f;
-        float g = 0.f;
-        for (int e = nbr_ptr[pos[r]]; e < nbr_ptr[pos[r] + 1]; ++e)
-            g += msg[((size_t)nbr_slot[e] * S + st[r]) * kD + lane];
-        A[r * KF + lane] = g;
+        st[r] = (r == 0 || last_live) ? s0 + r : s0;
+        x[r] = lane < F ? xs[(q * nb + st[r]) * F + lane] : 0.f;
+        acc[r] = 0.f;
     }
+    const int e0 = nbr_ptr[pos], e1 = nbr_ptr[pos + 1];
+    const int slot = own_slot[pos];
+    const int v = order[pos];
+    for (int e = e0; e < e1; ++e) {
+        const int base = nbr_slot[e] * S;
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] += msg[(base + st[r]) * kD + lane];
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) A[r * KF + lane] = acc[r];
     __syncwarp();
     matvec<R, kD>(w.g1, w.bg1, A, KF, acc);
 #pragma unroll
     for (int r = 0; r < R; ++r) Bf[r * KF + lane] = fmaxf(acc[r], 0.f);
     __syncwarp();
     matvec<R, kD>(w.g2, w.bg2, Bf, KF, acc);
-    bool any = false;
-    int slot[R];
+    float *hrow = H + ((size_t)v * B + b_first + s0) * kD + lane;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         acc[r] = fmaxf(acc[r], 0.f);
-        if (live[r]) H[((size_t)order[pos[r]] * B + b_first + st[r]) * kD + lane] = acc[r];
-        slot[r] = own_slot[pos[r]];
-        any |= slot[r] >= 0;
+        if (r == 0 || last_live) hrow[r * kD] = acc[r];
     }
-    if (!any) return;                       // nobody consumes these messages (warp-uniform)
+    if (slot < 0) return;                   // nobody consumes this node's message
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         A[r * KF + lane] = acc[r];
@@ -130,8 +128,7 @@ __device__ __forceinline__ void run_rows(const Weights32 &w, const float (&wf1)[
     matvec<R, kD>(w.f2, w.bf2, Bf, KF, acc);
 #pragma unroll
     for (int r = 0; r < R; ++r)
-        if (live[r] && slot[r] >= 0)
-            msg[((size_t)slot[r] * S + st[r]) * kD + lane] = fmaxf(acc[r], 0.f);
+        if (r == 0 || last_live) msg[((slot * S) + st[r]) * kD + lane] = fmaxf(acc[r], 0.f);
 }
 
 template <int F4>   // feature width padded to 4 * F4
@@ -217,15 +214,22 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         const int p0 = level_ptr[level];
         const int rows = (level_ptr[level + 1] - p0) * nb;
         const float *xs = xstage + (size_t)(level & 1) * p.x_floats;
+        const int width = level_ptr[level + 1] - p0;
         if (rows <= kWarps) {
             // narrow level: one row per warp, shortest dependent chains
-            if (warp < rows)
-                run_rows<1, KF>(w, wf1, warp, rows, p0, nb, p.S, F, lane, order, nbr_ptr, nbr_slot,
-                                own_slot, msg, xs, H, B, b_first, A, Bf);
+            if (warp < rows) {
+                const int q = warp / nb, s0 = warp - q * nb;
+                run_node<1, KF>(w, wf1, p0 + q, q, s0, true, nb, p.S, F, lane, order, nbr_ptr,
+                                nbr_slot, own_slot, msg, xs, H, B, b_first, A, Bf);
+            }
         } else {
-            for (int r = 2 * warp; r < rows; r += 2 * kWarps)
-                run_rows<2, KF>(w, wf1, r, rows, p0, nb, p.S, F, lane, order, nbr_ptr, nbr_slot,
-                                own_slot, msg, xs, H, B, b_first, A, Bf);
+            // two states of one node per warp pass
+            const int ppn = (nb + 1) >> 1;
+            for (int item = warp; item < width * ppn; item += kWarps) {
+                const int q = item / ppn, s0 = (item - q * ppn) * 2;
+                run_node<2, KF>(w, wf1, p0 + q, q, s0, s0 + 1 < nb, nb, p.S, F, lane, order,
+                                nbr_ptr, nbr_slot, own_slot, msg, xs, H, B, b_first, A, Bf);
+            }
         }
         __pipeline_wait_prior(0);
         __syncthreads();

@@ -20,6 +20,7 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
     __shared__ uint8_t s_dev[kTile][kTile + 4];
     __shared__ uint8_t s_placed[kTile][kTile + 4];
     __shared__ int s_cur[kTile];
+    __shared__ float s_cost[kTile], s_bytes[kTile];
     const int v0 = blockIdx.x * kTile, b0 = blockIdx.y * kTile;
     const int F = m + 4;
     for (int i = threadIdx.x; i < kTile * kTile; i += blockDim.x) {
@@ -30,12 +31,16 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
         s_placed[bl][vl] = ok ? placed[(size_t)b * n + v] : 0;
     }
     if (threadIdx.x < kTile) s_cur[threadIdx.x] = (b0 + threadIdx.x < B) ? cur[b0 + threadIdx.x] : -1;
+    if (threadIdx.x >= 32 && threadIdx.x < 32 + kTile && v0 + threadIdx.x - 32 < n) {
+        s_cost[threadIdx.x - 32] = cost[v0 + threadIdx.x - 32];
+        s_bytes[threadIdx.x - 32] = bytes[v0 + threadIdx.x - 32];
+    }
     __syncthreads();
     const int nb = min(kTile, B - b0);
     const int nv = min(kTile, n - v0);
     for (int vl = 0; vl < nv; ++vl) {
         const int v = v0 + vl;
-        const float c = cost[v], s = bytes[v];
+        const float c = s_cost[vl], s = s_bytes[vl];
         float *out = X + ((size_t)v * B + b0) * F;
         for (int i = threadIdx.x; i < nb * F; i += blockDim.x) {
             const int bl = i / F, k = i - bl * F;

@@ -8,7 +8,7 @@
 // partial sums of l_i(e_u) (one warp per state, lanes over the output columns,
 // the set of each node read from the relation row of c). Kernel 2 adds the
 // chunks in a fixed order (deterministic, no atomics), applies h_i, the head and
-// the softmax, one block per state.
+// the softmax, eight states per block so that each weight is read once per block.
 #include <algorithm>
 #include <cmath>
 
@@ -21,7 +21,8 @@ namespace {
 constexpr int kPoolThreads = 256;
 constexpr int kPoolWarps = kPoolThreads / 32;
 constexpr int kMaxCols = PLACETO_MAX_D / 32;   // output columns per lane
-constexpr int kHeadThreads = 128;
+constexpr int kHeadThreads = 256;
+constexpr int kHeadStates = 8;      // states finished per block of the head kernel
 
 struct PoolPlan {
     int states_per_block;
@@ -123,81 +124,120 @@ pool_partial_kernel(const PoolArgs a, const PoolPlan p) {
     }
 }
 
-// y[0..out) = act(bias + v W) with the whole block; v, y in shared memory.
-__device__ __forceinline__ void block_dense(const float *__restrict__ W,
-                                            const float *__restrict__ bias, int in, int out,
-                                            bool relu, const float *v, float *y) {
+// dst[s][0..out) = act(bias + src[s][0..in) W) for the kHeadStates rows of a block.
+// Wide layers: one thread per output column carries all rows, so each weight is
+// read once per block (coalesced over columns) with several loads in flight.
+// Narrow layers (the device logits): one warp per (row, column), the lanes split
+// the inner dimension and combine with a shuffle reduction.
+__device__ __forceinline__ void head_dense(const float *__restrict__ W,
+                                           const float *__restrict__ bias, int in, int out,
+                                           bool relu, const float *src, int src_stride, float *dst,
+                                           int dst_stride) {
     if (out >= 32) {
         for (int j = threadIdx.x; j < out; j += blockDim.x) {
-            float s = bias[j];
-            for (int k = 0; k < in; ++k) s = fmaf(v[k], W[(size_t)k * out + j], s);
-            y[j] = relu ? fmaxf(s, 0.f) : s;
+            float acc[kHeadStates];
+            const float b = bias[j];
+#pragma unroll
+            for (int s = 0; s < kHeadStates; ++s) acc[s] = b;
+            int k = 0;
+            for (; k + 4 <= in; k += 4) {
+                const float w0 = W[(size_t)k * out + j], w1 = W[(size_t)(k + 1) * out + j];
+                const float w2 = W[(size_t)(k + 2) * out + j], w3 = W[(size_t)(k + 3) * out + j];
+#pragma unroll
+                for (int s = 0; s < kHeadStates; ++s) {
+                    const float *v = src + s * src_stride + k;
+                    acc[s] = fmaf(v[0], w0, acc[s]);
+                    acc[s] = fmaf(v[1], w1, acc[s]);
+                    acc[s] = fmaf(v[2], w2, acc[s]);
+                    acc[s] = fmaf(v[3], w3, acc[s]);
+                }
+            }
+            for (; k < in; ++k) {
+                const float w0 = W[(size_t)k * out + j];
+#pragma unroll
+                for (int s = 0; s < kHeadStates; ++s)
+                    acc[s] = fmaf(src[s * src_stride + k], w0, acc[s]);
+            }
+#pragma unroll
+            for (int s = 0; s < kHeadStates; ++s)
+                dst[s * dst_stride + j] = relu ? fmaxf(acc[s], 0.f) : acc[s];
         }
     } else {
-        // few outputs (the device logits): one warp per output, lanes split the
-        // inner dimension and combine with a shuffle reduction
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-        for (int j = warp; j < out; j += nw) {
-            float s = 0.f;
-            for (int k = lane; k < in; k += 32) s = fmaf(v[k], W[(size_t)k * out + j], s);
+        for (int item = warp; item < out * kHeadStates; item += nw) {
+            const int s = item / out, j = item - s * out;
+            float acc = 0.f;
+            for (int k = lane; k < in; k += 32)
+                acc = fmaf(src[s * src_stride + k], W[(size_t)k * out + j], acc);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            s += bias[j];
-            if (lane == 0) y[j] = relu ? fmaxf(s, 0.f) : s;
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            acc += bias[j];
+            if (lane == 0) dst[s * dst_stride + j] = relu ? fmaxf(acc, 0.f) : acc;
         }
     }
     __syncthreads();
 }
 
-__device__ __forceinline__ float *block_mlp(const DevMlp &net, const float *in, float *tmp,
-                                            float *out) {
+__device__ __forceinline__ void head_mlp(const DevMlp &net, const float *in, int in_stride,
+                                         float *tmp, int tmp_stride, float *out, int out_stride) {
     const bool relu = net.act == 0;
     if (net.n_layers == 1) {
-        block_dense(net.W1, net.b1, net.in_dim, net.out_dim, relu && net.final_act, in, out);
-        return out;
+        head_dense(net.W1, net.b1, net.in_dim, net.out_dim, relu && net.final_act, in, in_stride,
+                   out, out_stride);
+        return;
     }
-    block_dense(net.W1, net.b1, net.in_dim, net.hidden_dim, relu, in, tmp);
-    block_dense(net.W2, net.b2, net.hidden_dim, net.out_dim, relu && net.final_act, tmp, out);
-    return out;
+    head_dense(net.W1, net.b1, net.in_dim, net.hidden_dim, relu, in, in_stride, tmp, tmp_stride);
+    head_dense(net.W2, net.b2, net.hidden_dim, net.out_dim, relu && net.final_act, tmp, tmp_stride,
+               out, out_stride);
 }
 
+// One block finishes kHeadStates states: chunk partial sums -> h_i -> head -> softmax.
 __global__ void __launch_bounds__(kHeadThreads)
 pool_head_kernel(const PoolArgs a, int tmp_floats) {
     extern __shared__ __align__(16) float smem[];
     const int d = a.d, F = a.F, B = a.B, m = a.m;
     const int E = 2 * d + F, Z = 5 * d + F;
-    float *z = smem;                      // [Z]
-    float *sum = z + ((Z + 3) & ~3);      // [3][d]
-    float *tmp = sum + 3 * d;             // [tmp_floats] hidden rows
-    float *lg = tmp + tmp_floats;         // [m]
-    const int b = blockIdx.x;
-    const int c = a.cur[b];
-    const bool valid = c >= 0 && c < a.n;
-    for (int j = threadIdx.x; j < 3 * d; j += blockDim.x) {
-        float s = 0.f;
-        for (int ch = 0; ch < a.chunks; ++ch) s += a.partial[((size_t)ch * B + b) * 3 * d + j];
-        sum[j] = s;
+    const int Zs = (Z + 3) & ~3;
+    float *z = smem;                               // [states][Zs]
+    float *sum = z + kHeadStates * Zs;             // [states][3 d]
+    float *tmp = sum + kHeadStates * 3 * d;        // [states][tmp_floats]
+    float *lg = tmp + kHeadStates * tmp_floats;    // [states][m]
+    const int b0 = blockIdx.x * kHeadStates;
+    for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
+        const int s = i / (3 * d), j = i - s * 3 * d;
+        const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
+        float acc = 0.f;
+        for (int ch = 0; ch < a.chunks; ++ch) acc += a.partial[((size_t)ch * B + b) * 3 * d + j];
+        sum[i] = acc;
     }
-    if (valid) {
-        for (int k = threadIdx.x; k < E; k += blockDim.x)
-            z[k] = k < d ? a.H[0][((size_t)c * B + b) * d + k]
-                 : k < 2 * d ? a.H[1][((size_t)c * B + b) * d + (k - d)]
-                             : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
-    } else {
-        for (int k = threadIdx.x; k < E; k += blockDim.x) z[k] = nanf("");
+    for (int i = threadIdx.x; i < kHeadStates * E; i += blockDim.x) {
+        const int s = i / E, k = i - s * E;
+        const int b = min(b0 + s, B - 1);
+        const int c = a.cur[b];
+        float v = 0.f;
+        if (c >= 0 && c < a.n)
+            v = k < d ? a.H[0][((size_t)c * B + b) * d + k]
+              : k < 2 * d ? a.H[1][((size_t)c * B + b) * d + (k - d)]
+                          : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
+        z[s * Zs + k] = v;
     }
     __syncthreads();
-    for (int i = 0; i < 3; ++i) block_mlp(a.h[i], sum + i * d, tmp, z + E + i * d);
-    block_mlp(a.head, z, tmp, lg);
-    if (threadIdx.x == 0) {
-        float mx = lg[0];
-        for (int k = 1; k < m; ++k) mx = fmaxf(mx, lg[k]);
+    for (int i = 0; i < 3; ++i)
+        head_mlp(a.h[i], sum + i * d, 3 * d, tmp, tmp_floats, z + E + i * d, Zs);
+    head_mlp(a.head, z, Zs, tmp, tmp_floats, lg, m);
+    if (threadIdx.x < kHeadStates && b0 + threadIdx.x < B) {
+        const int b = b0 + threadIdx.x;
+        const float *l = lg + threadIdx.x * m;
+        const int c = a.cur[b];
+        // a current node out of range yields NaN (ReLU would swallow a NaN input)
+        const bool valid = c >= 0 && c < a.n;
+        float mx = l[0];
+        for (int k = 1; k < m; ++k) mx = fmaxf(mx, l[k]);
         float tot = 0.f;
-        for (int k = 0; k < m; ++k) tot += expf(lg[k] - mx);
+        for (int k = 0; k < m; ++k) tot += expf(l[k] - mx);
         for (int k = 0; k < m; ++k) {
-            // a current node out of range yields NaN (ReLU would swallow a NaN input)
-            a.logits[(size_t)b * m + k] = valid ? lg[k] : nanf("");
-            if (a.probs) a.probs[(size_t)b * m + k] = valid ? expf(lg[k] - mx) / tot : nanf("");
+            a.logits[(size_t)b * m + k] = valid ? l[k] : nanf("");
+            if (a.probs) a.probs[(size_t)b * m + k] = valid ? expf(l[k] - mx) / tot : nanf("");
         }
     }
 }
@@ -248,12 +288,14 @@ cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
     for (int i = 0; i < 3; ++i)
         if (a.h[i].n_layers == 2) tmp_floats = std::max(tmp_floats, a.h[i].hidden_dim);
     tmp_floats = (tmp_floats + 3) & ~3;
-    const size_t head_smem = (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m + 4) * sizeof(float);
+    const size_t head_smem =
+        (size_t)kHeadStates * (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m) * sizeof(float) + 16;
     cudaError_t err = cudaFuncSetAttribute(pool_head_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)head_smem);
     if (err != cudaSuccess) return err;
-    pool_head_kernel<<<a.B, kHeadThreads, head_smem, stream>>>(a, tmp_floats);
+    const int blocks = (a.B + kHeadStates - 1) / kHeadStates;
+    pool_head_kernel<<<blocks, kHeadThreads, head_smem, stream>>>(a, tmp_floats);
     count_launch();
     return cudaGetLastError();
 }
