@@ -21,7 +21,7 @@ namespace {
 constexpr int kPoolThreads = 256;
 constexpr int kPoolWarps = kPoolThreads / 32;
 constexpr int kMaxCols = PLACETO_MAX_D / 32;   // output columns per lane
-constexpr int kHeadThreads = 256;
+constexpr int kHeadThreads = 512;
 constexpr int kHeadStates = 8;      // states finished per block of the head kernel
 
 struct PoolPlan {
@@ -125,42 +125,70 @@ pool_partial_kernel(const PoolArgs a, const PoolPlan p) {
 }
 
 // dst[s][0..out) = act(bias + src[s][0..in) W) for the kHeadStates rows of a block.
-// Wide layers: one thread per output column carries all rows, so each weight is
-// read once per block (coalesced over columns) with several loads in flight.
-// Narrow layers (the device logits): one warp per (row, column), the lanes split
-// the inner dimension and combine with a shuffle reduction.
+// Wide layers: a thread owns one output column and one part of the inner
+// dimension for all rows, so each weight is read once per block (coalesced over
+// columns) with eight loads in flight; the parts are then added in a fixed order
+// through `red`. Narrow layers (the device logits): one warp per (row, column),
+// the lanes split the inner dimension and combine with a shuffle reduction.
 __device__ __forceinline__ void head_dense(const float *__restrict__ W,
                                            const float *__restrict__ bias, int in, int out,
                                            bool relu, const float *src, int src_stride, float *dst,
-                                           int dst_stride) {
+                                           int dst_stride, float *red) {
     if (out >= 32) {
-        for (int j = threadIdx.x; j < out; j += blockDim.x) {
-            float acc[kHeadStates];
-            const float b = bias[j];
+        // parts * out <= blockDim.x, so `red` (blockDim.x * kHeadStates floats) holds
+        // every partial product; layers wider than the block take several column passes
+        const int parts = max(1, min((int)blockDim.x / out, (in + 7) / 8));
+        const int per = ((in + parts - 1) / parts + 3) & ~3;
+        const bool vec = (reinterpret_cast<uintptr_t>(src) & 15) == 0 && (src_stride & 3) == 0;
+        for (int j0 = 0; j0 < out; j0 += blockDim.x) {
+            const int cols = min(out - j0, (int)blockDim.x);
+            const int part = threadIdx.x / cols, jl = threadIdx.x - part * cols;
+            const int j = j0 + jl;
+            if (part < parts) {
+                float acc[kHeadStates];
 #pragma unroll
-            for (int s = 0; s < kHeadStates; ++s) acc[s] = b;
-            int k = 0;
-            for (; k + 4 <= in; k += 4) {
-                const float w0 = W[(size_t)k * out + j], w1 = W[(size_t)(k + 1) * out + j];
-                const float w2 = W[(size_t)(k + 2) * out + j], w3 = W[(size_t)(k + 3) * out + j];
+                for (int s = 0; s < kHeadStates; ++s) acc[s] = 0.f;
+                const int k1 = min(in, (part + 1) * per);
+                int k = part * per;
+                for (; k + 8 <= k1; k += 8) {
+                    float wv[8];
 #pragma unroll
-                for (int s = 0; s < kHeadStates; ++s) {
-                    const float *v = src + s * src_stride + k;
-                    acc[s] = fmaf(v[0], w0, acc[s]);
-                    acc[s] = fmaf(v[1], w1, acc[s]);
-                    acc[s] = fmaf(v[2], w2, acc[s]);
-                    acc[s] = fmaf(v[3], w3, acc[s]);
+                    for (int t = 0; t < 8; ++t) wv[t] = W[(size_t)(k + t) * out + j];
+#pragma unroll
+                    for (int s = 0; s < kHeadStates; ++s) {
+                        const float *v = src + s * src_stride + k;
+                        float4 v0, v1;
+                        if (vec) {
+                            v0 = *reinterpret_cast<const float4 *>(v);
+                            v1 = *reinterpret_cast<const float4 *>(v + 4);
+                        } else {
+                            v0 = make_float4(v[0], v[1], v[2], v[3]);
+                            v1 = make_float4(v[4], v[5], v[6], v[7]);
+                        }
+                        acc[s] = fmaf(v0.x, wv[0], acc[s]); acc[s] = fmaf(v0.y, wv[1], acc[s]);
+                        acc[s] = fmaf(v0.z, wv[2], acc[s]); acc[s] = fmaf(v0.w, wv[3], acc[s]);
+                        acc[s] = fmaf(v1.x, wv[4], acc[s]); acc[s] = fmaf(v1.y, wv[5], acc[s]);
+                        acc[s] = fmaf(v1.z, wv[6], acc[s]); acc[s] = fmaf(v1.w, wv[7], acc[s]);
+                    }
                 }
-            }
-            for (; k < in; ++k) {
-                const float w0 = W[(size_t)k * out + j];
+                for (; k < k1; ++k) {
+                    const float w0 = W[(size_t)k * out + j];
+#pragma unroll
+                    for (int s = 0; s < kHeadStates; ++s)
+                        acc[s] = fmaf(src[s * src_stride + k], w0, acc[s]);
+                }
 #pragma unroll
                 for (int s = 0; s < kHeadStates; ++s)
-                    acc[s] = fmaf(src[s * src_stride + k], w0, acc[s]);
+                    red[(part * kHeadStates + s) * cols + jl] = acc[s];
             }
-#pragma unroll
-            for (int s = 0; s < kHeadStates; ++s)
-                dst[s * dst_stride + j] = relu ? fmaxf(acc[s], 0.f) : acc[s];
+            __syncthreads();
+            for (int i = threadIdx.x; i < kHeadStates * cols; i += blockDim.x) {
+                const int s = i / cols, jj = i - s * cols;
+                float acc = bias[j0 + jj];
+                for (int q = 0; q < parts; ++q) acc += red[(q * kHeadStates + s) * cols + jj];
+                dst[s * dst_stride + j0 + jj] = relu ? fmaxf(acc, 0.f) : acc;
+            }
+            __syncthreads();
         }
     } else {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -178,17 +206,25 @@ __device__ __forceinline__ void head_dense(const float *__restrict__ W,
     __syncthreads();
 }
 
+// Asks for `count` floats to be brought into L2 (the block's threads share the lines).
+__device__ __forceinline__ void prefetch_l2(const float *p, size_t count) {
+    const char *base = reinterpret_cast<const char *>(p);
+    for (size_t off = (size_t)threadIdx.x * 128; off < count * sizeof(float); off += (size_t)blockDim.x * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+}
+
 __device__ __forceinline__ void head_mlp(const DevMlp &net, const float *in, int in_stride,
-                                         float *tmp, int tmp_stride, float *out, int out_stride) {
+                                         float *tmp, int tmp_stride, float *out, int out_stride,
+                                         float *red) {
     const bool relu = net.act == 0;
     if (net.n_layers == 1) {
         head_dense(net.W1, net.b1, net.in_dim, net.out_dim, relu && net.final_act, in, in_stride,
-                   out, out_stride);
+                   out, out_stride, red);
         return;
     }
-    head_dense(net.W1, net.b1, net.in_dim, net.hidden_dim, relu, in, in_stride, tmp, tmp_stride);
+    head_dense(net.W1, net.b1, net.in_dim, net.hidden_dim, relu, in, in_stride, tmp, tmp_stride, red);
     head_dense(net.W2, net.b2, net.hidden_dim, net.out_dim, relu && net.final_act, tmp, tmp_stride,
-               out, out_stride);
+               out, out_stride, red);
 }
 
 // One block finishes kHeadStates states: chunk partial sums -> h_i -> head -> softmax.
@@ -202,7 +238,11 @@ pool_head_kernel(const PoolArgs a, int tmp_floats) {
     float *sum = z + kHeadStates * Zs;             // [states][3 d]
     float *tmp = sum + kHeadStates * 3 * d;        // [states][tmp_floats]
     float *lg = tmp + kHeadStates * tmp_floats;    // [states][m]
+    float *red = lg + ((kHeadStates * m + 3) & ~3);   // [blockDim.x * states] partial products
     const int b0 = blockIdx.x * kHeadStates;
+    prefetch_l2(a.head.W1, (size_t)a.head.in_dim * a.head.hidden_dim);
+    if (a.head.n_layers == 2) prefetch_l2(a.head.W2, (size_t)a.head.hidden_dim * a.head.out_dim);
+    for (int i = 0; i < 3; ++i) prefetch_l2(a.h[i].W1, (size_t)a.h[i].in_dim * a.h[i].hidden_dim);
     for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
         const int s = i / (3 * d), j = i - s * 3 * d;
         const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
@@ -223,8 +263,8 @@ pool_head_kernel(const PoolArgs a, int tmp_floats) {
     }
     __syncthreads();
     for (int i = 0; i < 3; ++i)
-        head_mlp(a.h[i], sum + i * d, 3 * d, tmp, tmp_floats, z + E + i * d, Zs);
-    head_mlp(a.head, z, Zs, tmp, tmp_floats, lg, m);
+        head_mlp(a.h[i], sum + i * d, 3 * d, tmp, tmp_floats, z + E + i * d, Zs, red);
+    head_mlp(a.head, z, Zs, tmp, tmp_floats, lg, m, red);
     if (threadIdx.x < kHeadStates && b0 + threadIdx.x < B) {
         const int b = b0 + threadIdx.x;
         const float *l = lg + threadIdx.x * m;
@@ -289,7 +329,8 @@ cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
         if (a.h[i].n_layers == 2) tmp_floats = std::max(tmp_floats, a.h[i].hidden_dim);
     tmp_floats = (tmp_floats + 3) & ~3;
     const size_t head_smem =
-        (size_t)kHeadStates * (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m) * sizeof(float) + 16;
+        ((size_t)kHeadStates * (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m) + 4 +
+         (size_t)kHeadThreads * kHeadStates) * sizeof(float);
     cudaError_t err = cudaFuncSetAttribute(pool_head_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)head_smem);
