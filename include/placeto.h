@@ -49,7 +49,9 @@ typedef enum {
     PLACETO_ERR_WORKSPACE = 3,   /* workspace smaller than placeto_workspace_bytes() */
     PLACETO_ERR_UNSUPPORTED = 4, /* dimensions beyond the limits below, or flag not applicable */
     PLACETO_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
-    PLACETO_ERR_NO_MEMORY = 6    /* host or device allocation failed in graph_create */
+    PLACETO_ERR_NO_MEMORY = 6,   /* host or device allocation failed in graph_create */
+    PLACETO_ERR_SCRATCH_LIMIT = 7 /* batch too large for the built-in scratch of
+                                     placeto_policy_logits_static */
 } placeto_status;
 
 /* Limits of this build. */
@@ -229,6 +231,41 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
                                            const uint8_t *placed, int32_t B, float *logits,
                                            float *probs, void *workspace, size_t workspace_bytes,
                                            uint32_t flags, void *stream);
+
+/*
+ * placeto_policy_logits without a workspace argument, for callers that must not
+ * allocate device memory. (The paper has no counterpart: this is a deployment
+ * variant of the call above, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving
+ * loop with a frozen memory budget, in a plug-in whose host application owns the
+ * allocator, or in a process that must not trigger the implicit device
+ * synchronisation that an allocation causes. Such a caller still passes every
+ * input and output buffer (X, H_down, H_up, cur, logits, probs), exactly as for
+ * placeto_policy_logits; only the chunk partial sums of step 3, which the normal
+ * call keeps in the caller's workspace, live instead in an array that is part of
+ * the library image: PLACETO_STATIC_SCRATCH_BYTES bytes of device memory on every
+ * GPU that loads the library, held until the process exits.
+ *
+ * Limits and rules
+ *   - The partial sums need chunks * B * 3 * d floats (chunks grows with n). If that
+ *     exceeds PLACETO_STATIC_SCRATCH_BYTES the call returns PLACETO_ERR_SCRATCH_LIMIT
+ *     and launches nothing; use placeto_policy_logits with a workspace then.
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating
+ *     library routine. The first call on each device looks up the array's device
+ *     address (a one-time set-up); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left there. Nothing in it has to start at zero: each call writes every
+ *     entry before reading it. Two calls that overlap on the GPU (different streams,
+ *     or different host threads) would overwrite each other's sums: serialise them.
+ *   - Results are identical to placeto_policy_logits for the same arguments and flags.
+ */
+#define PLACETO_STATIC_SCRATCH_BYTES (4u << 20)
+placeto_status placeto_policy_logits_static(const placeto_graph *g, const placeto_weights *w,
+                                            const float *X, const float *H_down,
+                                            const float *H_up, const int32_t *cur, int32_t B,
+                                            float *logits, float *probs, uint32_t flags,
+                                            void *stream);
 
 /* Number of kernels the most recent forward call of this thread launched (for accounting). */
 int32_t placeto_last_launch_count(void);

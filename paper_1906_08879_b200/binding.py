@@ -26,7 +26,8 @@ EXPORTS = (
     "placeto_status_string", "placeto_graph_create", "placeto_graph_info",
     "placeto_graph_host_view", "placeto_graph_destroy", "placeto_workspace_bytes",
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
-    "placeto_policy_forward", "placeto_policy_forward_host", "placeto_last_launch_count",
+    "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
+    "placeto_last_launch_count",
 )
 
 
@@ -72,7 +73,8 @@ def _load() -> ctypes.CDLL:
     lib.placeto_last_launch_count.restype = ctypes.c_int32
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
-                 "placeto_policy_forward", "placeto_policy_forward_host"):
+                 "placeto_policy_forward", "placeto_policy_forward_host",
+                 "placeto_policy_logits_static"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -287,6 +289,25 @@ def placeto_policy_forward_host(g: Graph, w: Weights, cost, nbytes, dev, cur, pl
                                             _p(logits), _p(probs), _p(ws),
                                             ctypes.c_size_t(ws.numel()), ctypes.c_uint32(flags),
                                             _stream(stream)), "placeto_policy_forward_host")
+    return logits, probs
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def placeto_policy_logits_static(g: Graph, w: Weights, X, H_down, H_up, cur, logits, probs=None,
+                                 flags: int = 0, stream=None):
+    """placeto_policy_logits for callers that may not allocate device memory:
+    no workspace argument, the chunk partial sums live in an array built into
+    the library (STATIC_SCRATCH_BYTES per GPU). This wrapper allocates nothing
+    either, so `logits` (and `probs`, if wanted) must be passed in. Raises
+    PlacetoError with status 7 when the batch needs more scratch than the array
+    holds. Calls on one device share that array: do not let two overlap."""
+    B = X.shape[1]
+    _check(_lib.placeto_policy_logits_static(g.handle, ctypes.byref(w.c), _p(X), _p(H_down),
+                                             _p(H_up), _p(cur), ctypes.c_int32(B), _p(logits),
+                                             _p(probs), ctypes.c_uint32(flags), _stream(stream)),
+           "placeto_policy_logits_static")
     return logits, probs
 
 

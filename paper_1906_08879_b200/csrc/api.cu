@@ -3,6 +3,7 @@
 // happens on the host.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "kernels.cuh"
@@ -186,6 +187,36 @@ placeto_status common_checks(const placeto_graph *g, int32_t B, const void *ws, 
 }
 
 }  // namespace
+
+// Scratch of placeto_policy_logits_static: part of the library image, one copy
+// per device that loads it. In host code the symbol below is only a handle: the
+// address a kernel can use comes from cudaGetSymbolAddress, looked up once per
+// device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[PLACETO_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+char *g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device`, or nullptr on failure.
+char *static_scratch_address(int device) {
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_ptr[device]) return g_scratch_ptr[device];
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return nullptr;
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) return nullptr;
+    void *ptr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (prev != device) cudaSetDevice(prev);
+    if (e != cudaSuccess || !ptr) return nullptr;
+    g_scratch_ptr[device] = static_cast<char *>(ptr);
+    return g_scratch_ptr[device];
+}
+
+}  // namespace
 }  // namespace placeto
 
 extern "C" {
@@ -199,6 +230,7 @@ const char *placeto_status_string(placeto_status s) {
         case PLACETO_ERR_UNSUPPORTED: return "unsupported dimensions or flag";
         case PLACETO_ERR_CUDA: return "CUDA error";
         case PLACETO_ERR_NO_MEMORY: return "out of memory";
+        case PLACETO_ERR_SCRATCH_LIMIT: return "batch exceeds the built-in scratch of the no-allocation call";
     }
     return "unknown status";
 }
@@ -456,6 +488,29 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     if (probs && cudaMemcpyAsync(probs, d_probs, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return PLACETO_ERR_CUDA;
     return cuda_status(cudaStreamSynchronize(st));
+}
+
+placeto_status placeto_policy_logits_static(const placeto_graph *g, const placeto_weights *w,
+                                            const float *X, const float *H_down,
+                                            const float *H_up, const int32_t *cur, int32_t B,
+                                            float *logits, float *probs, uint32_t flags,
+                                            void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1 || !flags_ok(flags)) return PLACETO_ERR_INVALID_ARG;
+    if ((size_t)B * g->host.n > (size_t)1 << 31) return PLACETO_ERR_UNSUPPORTED;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_LOGITS);   // partial sums sit at offset 0
+    if (L.total > PLACETO_STATIC_SCRATCH_BYTES) return PLACETO_ERR_SCRATCH_LIMIT;
+    if (!X || !H_down || !H_up || !cur || !logits) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(H_down) || !aligned16(H_up) || !aligned16(cur) ||
+        !aligned16(logits) || (probs && !aligned16(probs)))
+        return PLACETO_ERR_INVALID_ARG;
+    char *scratch = static_scratch_address(g->device);
+    if (!scratch) return PLACETO_ERR_CUDA;
+    return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, scratch, L, flags,
+                    static_cast<cudaStream_t>(stream));
 }
 
 int32_t placeto_last_launch_count(void) { return t_launches; }
