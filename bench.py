@@ -78,6 +78,20 @@ def flops_pool(cfg):
     return 2.0 * (2 * d * d + d * F) * cfg["n"] * cfg["B"]
 
 
+def job_throughput(local_ms: float, states_per_rank: int, steps: int, dist=None, device="cpu"):
+    """Whole-job evaluations/s: every rank processed `states_per_rank` states per
+    step; the job takes as long as its slowest rank (max over ranks of the
+    device time). Returns (value, slowest_ms)."""
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    world = 1
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        world = dist.get_world_size()
+    slowest = float(t.item())
+    return states_per_rank * world * steps / (slowest * 1e-3), slowest
+
+
 # ------------------------------------------------------------ CPU checker ---
 
 def time_oracle(cfg, budget_s: float, threads: int):
@@ -252,11 +266,7 @@ def run_b200(args):
     total_ms, launches = timed(step, args.steps, count_launches=True)
     barrier()
     clocks = sampler.stop()
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
-    value = B * world * args.steps / (total_ms * 1e-3)
+    value, total_ms = job_throughput(total_ms, B, args.steps, dist, "cuda")
 
     # end to end through the host-buffer entry point: pinned inputs -> device -> results on host
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -272,10 +282,7 @@ def run_b200(args):
     barrier()
     e2e_ms, _ = timed(e2e_step, args.steps)
     barrier()
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = B * world * args.steps / (float(t.item()) * 1e-3)
+    e2e_value, _ = job_throughput(e2e_ms, B, args.steps, dist, "cuda")
     h2d = sum(x.numel() * x.element_size() for x in h_in)
     d2h = h_logits.numel() * 4 + h_probs.numel() * 4
     assert torch.equal(h_logits.cuda(), logits), "host and device entry points disagree"
