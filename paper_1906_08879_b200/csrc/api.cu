@@ -151,6 +151,10 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
         cudaError_t e = launch_embed_d32(a, g->info, stream);
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
+    if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d64_applicable(a)) {
+        cudaError_t e = launch_embed_d64(a, g->info, stream);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     return cuda_status(launch_embed_generic(a, g->info, schedule, stream));
 }
 

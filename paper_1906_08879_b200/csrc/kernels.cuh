@@ -89,6 +89,11 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
 bool embed_d32_applicable(const EmbedArgs &a);
 cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
+// embed_d64.cu: the same for d = 64 (four-warp column-split groups, both
+// directions in one block).
+bool embed_d64_applicable(const EmbedArgs &a);
+cudaError_t launch_embed_d64(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
+
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);
 cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
