@@ -76,7 +76,7 @@ placeto_status pool_weights_ok(const placeto_weights *w) {
 struct Layout {
     size_t msg[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
-    int chunks32, chunk_nodes32;   // and of the d = 32 kernel (0 when it cannot apply)
+    int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
 };
 
 // Workspace layout shared by every call; a call uses the leading part it needs.
@@ -92,8 +92,10 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         L.msg[0] = take(n * B * d * sizeof(float));
         L.msg[1] = take(n * B * d * sizeof(float));
     }
-    if (w->d == 32 && w->F >= 4 && w->F <= 16 && (w->F & 3) == 0)
-        pool_d32_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
+    if (w->F >= 4 && w->F <= 16 && (w->F & 3) == 0) {
+        if (w->d == 32) pool_d32_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
+        if (w->d == 64) pool_d64_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
+    }
     if (call == PLACETO_CALL_LOGITS || call >= PLACETO_CALL_FORWARD)
         L.partial = take((size_t)std::max(L.chunks, L.chunks32) * B * 3 * d * sizeof(float));
     if (call >= PLACETO_CALL_FORWARD) {
@@ -171,9 +173,10 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     a.partial = reinterpret_cast<float *>(ws + L.partial);
     a.logits = logits; a.probs = probs;
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d; a.m = w->m;
-    if (!(flags & PLACETO_GENERIC) && L.chunks32 > 0 && pool_d32_applicable(a)) {
+    const bool fast32 = pool_d32_applicable(a), fast64 = pool_d64_applicable(a);
+    if (!(flags & PLACETO_GENERIC) && L.chunks32 > 0 && (fast32 || fast64)) {
         a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
-        cudaError_t e = launch_pool_d32(a, g->info, stream);
+        cudaError_t e = fast32 ? launch_pool_d32(a, g->info, stream) : launch_pool_d64(a, g->info, stream);
         if (e == cudaSuccess) return cuda_status(launch_pool_head(a, stream));
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }

@@ -105,4 +105,9 @@ bool pool_d32_applicable(const PoolArgs &a);
 void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
 cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
+// policy_d64.cu: the same for d = 64 (weights of all three sets split over the block's warps)
+bool pool_d64_applicable(const PoolArgs &a);
+void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
+cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
+
 }  // namespace placeto

@@ -1,0 +1,182 @@
+// Step 3 of the policy (Sec. 2.2 step 3 of the Placeto paper) specialised for
+// d = 64 with single-layer ReLU l_i: partial sums over a chunk of nodes of
+//   l_i(e_u),   e_u = [h_down_u || h_up_u || x_u],   i = set of u relative to cur[b],
+// for a tile of states per block, in the layout the head kernel adds up.
+//
+// The three 140 x 64 matrices (with F = 12) are too large to switch per set, so
+// they stay resident, split over the block: eight warps, warp w owns output
+// columns [8w, 8w + 8), lane (quarter, col) keeps one quarter of the inner
+// dimension of its column for all three sets (3 x 36 registers). Every warp
+// walks all rows (state, node) of the block's tile: it reads its quarter of the
+// row from shared memory (broadcast 128-bit loads, 4 FMAs per load), combines
+// the quarters with two shuffles and adds relu(.) to the accumulator of the row's
+// set. Warps never synchronise after the tile is staged (cp.async). Summation
+// order is ascending node id per (chunk, state): deterministic.
+#include <cuda_pipeline.h>
+
+#include <algorithm>
+
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kD = 64;
+constexpr int kWarps = kD / 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kTileStates = 8;
+
+struct Pool64Plan {
+    int chunk_nodes, chunks;
+    size_t smem_bytes;
+};
+
+template <int KQ>
+__device__ __forceinline__ float quarter_dot(const float (&w)[KQ], const float *in) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int k = 0; k < KQ; k += 4) {
+        const float4 u = *reinterpret_cast<const float4 *>(in + k);
+        a0 = fmaf(u.x, w[k], a0);
+        a1 = fmaf(u.y, w[k + 1], a1);
+        a2 = fmaf(u.z, w[k + 2], a2);
+        a3 = fmaf(u.w, w[k + 3], a3);
+    }
+    float s = (a0 + a1) + (a2 + a3);
+    s += __shfl_xor_sync(0xffffffffu, s, 8);
+    s += __shfl_xor_sync(0xffffffffu, s, 16);
+    return s;
+}
+
+template <int F4>
+__global__ void __launch_bounds__(kThreads, 1)
+pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
+    constexpr int E = 2 * kD + 4 * F4;              // embedding row (features padded to 4 F4)
+    constexpr int KQ = ((E + 3) / 4 + 3) & ~3;      // inner width per lane quarter
+    constexpr int RS = 4 * KQ;                      // shared row stride (>= E, zero padded)
+    extern __shared__ __align__(16) float smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int quarter = lane >> 3, col = warp * 8 + (lane & 7);
+    const int n = a.n, B = a.B, F = a.F;
+    const int chunk = blockIdx.x;
+    const int u0 = chunk * p.chunk_nodes, nu = min(n, u0 + p.chunk_nodes) - u0;
+    const int b0 = blockIdx.y * kTileStates, nb = min(kTileStates, B - b0);
+
+    float *rows = smem;                                                    // [chunk][states][RS]
+    uint8_t *rel = reinterpret_cast<uint8_t *>(rows + (size_t)p.chunk_nodes * kTileStates * RS);
+                                                                           // [states][chunk]
+    // ---- stage the tile: every row as one contiguous [h_down | h_up | x | 0] vector
+    {
+        const int pieces = (2 * kD + F) / 4;            // 16-byte pieces per row (F multiple of 4)
+        for (int t = threadIdx.x; t < nu * nb * pieces; t += kThreads) {
+            const int r = t / pieces, k = (t - r * pieces) * 4;
+            const int q = r / nb, s = r - q * nb;
+            const size_t src = (size_t)(u0 + q) * B + b0 + s;
+            const float *from = k < kD ? a.H[0] + src * kD + k
+                              : k < 2 * kD ? a.H[1] + src * kD + (k - kD)
+                                           : a.X + src * F + (k - 2 * kD);
+            __pipeline_memcpy_async(rows + ((size_t)q * kTileStates + s) * RS + k, from, 16);
+        }
+        const int pad = RS - (2 * kD + F);
+        for (int t = threadIdx.x; t < nu * nb * pad; t += kThreads) {
+            const int r = t / pad, k = t - r * pad;
+            const int q = r / nb, s = r - q * nb;
+            rows[((size_t)q * kTileStates + s) * RS + 2 * kD + F + k] = 0.f;
+        }
+        for (int t = threadIdx.x; t < nb * nu; t += kThreads) {
+            const int s = t / nu, q = t - s * nu;
+            const int c = a.cur[b0 + s];
+            rel[s * p.chunk_nodes + q] = (c >= 0 && c < n) ? a.relation[(size_t)c * n + u0 + q] : 3;
+        }
+    }
+    // ---- this lane's weights: column `col`, its quarter of the inner dimension, three sets
+    float w0[KQ], w1[KQ], w2[KQ];
+#pragma unroll
+    for (int k = 0; k < KQ; ++k) {
+        const int kk = quarter * KQ + k;
+        const bool in_range = kk < 2 * kD + F;
+        w0[k] = in_range ? a.l[0].W1[kk * kD + col] : 0.f;
+        w1[k] = in_range ? a.l[1].W1[kk * kD + col] : 0.f;
+        w2[k] = in_range ? a.l[2].W1[kk * kD + col] : 0.f;
+    }
+    const float bias0 = a.l[0].b1[col], bias1 = a.l[1].b1[col], bias2 = a.l[2].b1[col];
+    __pipeline_commit();
+    __pipeline_wait_prior(0);
+    __syncthreads();
+
+    for (int s = 0; s < nb; ++s) {
+        float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f;
+        const uint8_t *rs = rel + s * p.chunk_nodes;
+        for (int q = 0; q < nu; ++q) {
+            const int set = rs[q];                               // warp-uniform
+            const float *in = rows + ((size_t)q * kTileStates + s) * RS + quarter * KQ;
+            if (set == 0) acc0 += fmaxf(quarter_dot<KQ>(w0, in) + bias0, 0.f);
+            else if (set == 1) acc1 += fmaxf(quarter_dot<KQ>(w1, in) + bias1, 0.f);
+            else if (set == 2) acc2 += fmaxf(quarter_dot<KQ>(w2, in) + bias2, 0.f);
+        }
+        if (quarter == 0) {
+            float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + col;
+            out[0] = acc0;
+            out[kD] = acc1;
+            out[2 * kD] = acc2;
+        }
+    }
+}
+
+bool relu1x64(const DevMlp &m, int in) {
+    return m.n_layers == 1 && m.in_dim == in && m.out_dim == kD && m.act == 0 && m.final_act == 1;
+}
+
+size_t tile_bytes(int chunk_nodes, int F) {
+    const int E = 2 * kD + F;
+    const int KQ = ((E + 3) / 4 + 3) & ~3;
+    return (size_t)chunk_nodes * kTileStates * 4 * KQ * sizeof(float) +
+           (((size_t)chunk_nodes * kTileStates + 15) & ~size_t(15));
+}
+
+}  // namespace
+
+bool pool_d64_applicable(const PoolArgs &a) {
+    if (a.d != kD || a.F < 4 || a.F > 16 || (a.F & 3)) return false;
+    for (int i = 0; i < 3; ++i)
+        if (!relu1x64(a.l[i], 2 * kD + a.F)) return false;
+    return true;
+}
+
+void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks) {
+    const size_t budget = (size_t)std::min(di.max_smem_optin, 227 * 1024) - 1024;
+    int cap = 1;
+    while (tile_bytes(cap + 1, F) <= budget) ++cap;
+    const int tiles = (B + kTileStates - 1) / kTileStates;
+    int c = (n + cap - 1) / cap;
+    if (c * tiles < di.sm_count) c = std::max(c, std::min(di.sm_count / tiles, (n + 7) / 8));
+    c = std::max(1, c);
+    *chunk_nodes = (n + c - 1) / c;
+    *chunks = (n + *chunk_nodes - 1) / *chunk_nodes;
+}
+
+cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+    Pool64Plan p;
+    p.chunk_nodes = a.chunk_nodes;
+    p.chunks = a.chunks;
+    p.smem_bytes = tile_bytes(p.chunk_nodes, a.F);
+    if (p.smem_bytes > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
+    void (*kern)(const PoolArgs, const Pool64Plan) = nullptr;
+    switch (a.F / 4) {
+        case 1: kern = pool_d64_kernel<1>; break;
+        case 2: kern = pool_d64_kernel<2>; break;
+        case 3: kern = pool_d64_kernel<3>; break;
+        case 4: kern = pool_d64_kernel<4>; break;
+        default: return cudaErrorNotSupported;
+    }
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)p.smem_bytes);
+    if (err != cudaSuccess) return err;
+    dim3 grid(p.chunks, (a.B + kTileStates - 1) / kTileStates);
+    kern<<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace placeto
