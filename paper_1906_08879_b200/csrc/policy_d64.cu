@@ -10,8 +10,10 @@
 // walks all rows (state, node) of the block's tile: it reads its quarter of the
 // row from shared memory (broadcast 128-bit loads, 4 FMAs per load), combines
 // the quarters with two shuffles and adds relu(.) to the accumulator of the row's
-// set. Warps never synchronise after the tile is staged (cp.async). Summation
-// order is ascending node id per (chunk, state): deterministic.
+// set. The rows of each (state, set) are compacted into index lists while the
+// tile is staged (cp.async), so the main loop runs set by set, two rows in
+// flight, without branching on the set. Warps never synchronise after staging.
+// Summation order is ascending node id per (chunk, state, set): deterministic.
 #include <cuda_pipeline.h>
 
 #include <algorithm>
@@ -32,21 +34,52 @@ struct Pool64Plan {
     size_t smem_bytes;
 };
 
-template <int KQ>
-__device__ __forceinline__ float quarter_dot(const float (&w)[KQ], const float *in) {
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+// Sum over one set's rows (node indices in `list`) of relu(bias + row . w), this
+// lane's column; two rows in flight, four accumulators each.
+template <int KQ, int RS>
+__device__ __forceinline__ float set_sum(const float (&w)[KQ], float bias, const uint8_t *list,
+                                         int count, const float *rows_s) {
+    float total = 0.f;
+    int i = 0;
+    for (; i + 2 <= count; i += 2) {
+        const float *in0 = rows_s + (size_t)list[i] * (kTileStates * RS);
+        const float *in1 = rows_s + (size_t)list[i + 1] * (kTileStates * RS);
+        float a[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-    for (int k = 0; k < KQ; k += 4) {
-        const float4 u = *reinterpret_cast<const float4 *>(in + k);
-        a0 = fmaf(u.x, w[k], a0);
-        a1 = fmaf(u.y, w[k + 1], a1);
-        a2 = fmaf(u.z, w[k + 2], a2);
-        a3 = fmaf(u.w, w[k + 3], a3);
+        for (int k = 0; k < KQ; k += 4) {
+            const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
+            const float4 v = *reinterpret_cast<const float4 *>(in1 + k);
+            a[0][0] = fmaf(u.x, w[k], a[0][0]);     a[1][0] = fmaf(v.x, w[k], a[1][0]);
+            a[0][1] = fmaf(u.y, w[k + 1], a[0][1]); a[1][1] = fmaf(v.y, w[k + 1], a[1][1]);
+            a[0][2] = fmaf(u.z, w[k + 2], a[0][2]); a[1][2] = fmaf(v.z, w[k + 2], a[1][2]);
+            a[0][3] = fmaf(u.w, w[k + 3], a[0][3]); a[1][3] = fmaf(v.w, w[k + 3], a[1][3]);
+        }
+        float s0 = (a[0][0] + a[0][1]) + (a[0][2] + a[0][3]);
+        float s1 = (a[1][0] + a[1][1]) + (a[1][2] + a[1][3]);
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, 8);
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+        total += fmaxf(s0 + bias, 0.f);
+        total += fmaxf(s1 + bias, 0.f);
     }
-    float s = (a0 + a1) + (a2 + a3);
-    s += __shfl_xor_sync(0xffffffffu, s, 8);
-    s += __shfl_xor_sync(0xffffffffu, s, 16);
-    return s;
+    if (i < count) {
+        const float *in0 = rows_s + (size_t)list[i] * (kTileStates * RS);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int k = 0; k < KQ; k += 4) {
+            const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
+            a0 = fmaf(u.x, w[k], a0);
+            a1 = fmaf(u.y, w[k + 1], a1);
+            a2 = fmaf(u.z, w[k + 2], a2);
+            a3 = fmaf(u.w, w[k + 3], a3);
+        }
+        float s0 = (a0 + a1) + (a2 + a3);
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+        total += fmaxf(s0 + bias, 0.f);
+    }
+    return total;
 }
 
 template <int F4>
@@ -64,8 +97,9 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     const int b0 = blockIdx.y * kTileStates, nb = min(kTileStates, B - b0);
 
     float *rows = smem;                                                    // [chunk][states][RS]
-    uint8_t *rel = reinterpret_cast<uint8_t *>(rows + (size_t)p.chunk_nodes * kTileStates * RS);
-                                                                           // [states][chunk]
+    // per state and set: the chunk's node indices of that set, ascending  [states][3][chunk]
+    uint8_t *lists = reinterpret_cast<uint8_t *>(rows + (size_t)p.chunk_nodes * kTileStates * RS);
+    __shared__ int counts[kTileStates][3];
     // ---- stage the tile: every row as one contiguous [h_down | h_up | x | 0] vector
     {
         const int pieces = (2 * kD + F) / 4;            // 16-byte pieces per row (F multiple of 4)
@@ -84,11 +118,25 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
             const int q = r / nb, s = r - q * nb;
             rows[((size_t)q * kTileStates + s) * RS + 2 * kD + F + k] = 0.f;
         }
-        for (int t = threadIdx.x; t < nb * nu; t += kThreads) {
-            const int s = t / nu, q = t - s * nu;
-            const int c = a.cur[b0 + s];
-            rel[s * p.chunk_nodes + q] = (c >= 0 && c < n) ? a.relation[(size_t)c * n + u0 + q] : 3;
+    }
+    if (warp < nb) {       // warp s compacts the relation row of its state into three lists
+        const int c = a.cur[b0 + warp];
+        const bool valid = c >= 0 && c < n;
+        const uint8_t *rel = a.relation + (size_t)(valid ? c : 0) * n + u0;
+        int cnt[3] = {0, 0, 0};
+        for (int base = 0; base < nu; base += 32) {
+            const int q = base + lane;
+            const int set = (valid && q < nu) ? rel[q] : 3;
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                const unsigned mask = __ballot_sync(0xffffffffu, set == i);
+                if (set == i)
+                    lists[(warp * 3 + i) * p.chunk_nodes + cnt[i] + __popc(mask & ((1u << lane) - 1))] =
+                        (uint8_t)q;
+                cnt[i] += __popc(mask);
+            }
         }
+        if (lane < 3) counts[warp][lane] = lane == 0 ? cnt[0] : (lane == 1 ? cnt[1] : cnt[2]);
     }
     // ---- this lane's weights: column `col`, its quarter of the inner dimension, three sets
     float w0[KQ], w1[KQ], w2[KQ];
@@ -106,15 +154,11 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     __syncthreads();
 
     for (int s = 0; s < nb; ++s) {
-        float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f;
-        const uint8_t *rs = rel + s * p.chunk_nodes;
-        for (int q = 0; q < nu; ++q) {
-            const int set = rs[q];                               // warp-uniform
-            const float *in = rows + ((size_t)q * kTileStates + s) * RS + quarter * KQ;
-            if (set == 0) acc0 += fmaxf(quarter_dot<KQ>(w0, in) + bias0, 0.f);
-            else if (set == 1) acc1 += fmaxf(quarter_dot<KQ>(w1, in) + bias1, 0.f);
-            else if (set == 2) acc2 += fmaxf(quarter_dot<KQ>(w2, in) + bias2, 0.f);
-        }
+        const float *rows_s = rows + (size_t)s * RS + quarter * KQ;
+        const uint8_t *ls = lists + (size_t)s * 3 * p.chunk_nodes;
+        const float acc0 = set_sum<KQ, RS>(w0, bias0, ls, counts[s][0], rows_s);
+        const float acc1 = set_sum<KQ, RS>(w1, bias1, ls + p.chunk_nodes, counts[s][1], rows_s);
+        const float acc2 = set_sum<KQ, RS>(w2, bias2, ls + 2 * p.chunk_nodes, counts[s][2], rows_s);
         if (quarter == 0) {
             float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + col;
             out[0] = acc0;
@@ -132,7 +176,7 @@ size_t tile_bytes(int chunk_nodes, int F) {
     const int E = 2 * kD + F;
     const int KQ = ((E + 3) / 4 + 3) & ~3;
     return (size_t)chunk_nodes * kTileStates * 4 * KQ * sizeof(float) +
-           (((size_t)chunk_nodes * kTileStates + 15) & ~size_t(15));
+           (((size_t)chunk_nodes * kTileStates * 3 + 15) & ~size_t(15));
 }
 
 }  // namespace
@@ -147,7 +191,7 @@ bool pool_d64_applicable(const PoolArgs &a) {
 void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks) {
     const size_t budget = (size_t)std::min(di.max_smem_optin, 227 * 1024) - 1024;
     int cap = 1;
-    while (tile_bytes(cap + 1, F) <= budget) ++cap;
+    while (cap < 255 && tile_bytes(cap + 1, F) <= budget) ++cap;
     const int tiles = (B + kTileStates - 1) / kTileStates;
     int c = (n + cap - 1) / cap;
     if (c * tiles < di.sm_count) c = std::max(c, std::min(di.sm_count / tiles, (n + 7) / 8));
@@ -161,7 +205,8 @@ cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_
     p.chunk_nodes = a.chunk_nodes;
     p.chunks = a.chunks;
     p.smem_bytes = tile_bytes(p.chunk_nodes, a.F);
-    if (p.smem_bytes > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
+    // node indices inside a chunk are stored as bytes
+    if (p.smem_bytes > (size_t)di.max_smem_optin || p.chunk_nodes > 255) return cudaErrorNotSupported;
     void (*kern)(const PoolArgs, const Pool64Plan) = nullptr;
     switch (a.F / 4) {
         case 1: kern = pool_d64_kernel<1>; break;
