@@ -156,6 +156,11 @@ typedef struct {
 #define PLACETO_COOPERATIVE 4u /* persistent cooperative launch: a level's nodes are spread over
                                   blocks, grid-wide sync between levels (small B, wide levels) */
 #define PLACETO_GENERIC 8u     /* use only the dimension-generic kernels (no specialised ones) */
+#define PLACETO_FMA_ONLY 16u   /* keep step 2 on the FP32 FMA pipes: do not use the tensor-core
+                                  kernel (TF32 head + tail split, three products per step) that
+                                  d = 64 otherwise takes */
+#define PLACETO_TENSOR 32u     /* use the tensor-core kernel of step 2 wherever it applies
+                                  (d = 32 or 64), also where the library would pick the FMA one */
 
 typedef enum {
     PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libplaceto.so")
 
 # flags and enums of placeto.h
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
+PLACETO_FMA_ONLY, PLACETO_TENSOR = 16, 32
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
 CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST = 0, 1, 2, 3
 

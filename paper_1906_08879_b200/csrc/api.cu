@@ -123,7 +123,8 @@ unsigned pick_schedule(unsigned flags) {
 }
 
 bool flags_ok(uint32_t flags) {
-    const uint32_t known = PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE | PLACETO_GENERIC;
+    const uint32_t known = PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE |
+                           PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR;
     if (flags & ~known) return false;
     const uint32_t sched = flags & (PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE);
     return (sched & (sched - 1)) == 0;   // at most one schedule
@@ -149,6 +150,11 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
     a.max_level_width = g->host.max_level_width;
     const unsigned schedule = pick_schedule(flags);
+    const bool want_mma = (flags & PLACETO_TENSOR) ? embed_mma_applicable(a) : embed_mma_preferred(a);
+    if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) && schedule == PLACETO_SLICED && want_mma) {
+        cudaError_t e = launch_embed_mma(a, g->info, stream);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d32_applicable(a)) {
         cudaError_t e = launch_embed_d32(a, g->info, stream);
         if (e != cudaErrorNotSupported) return cuda_status(e);

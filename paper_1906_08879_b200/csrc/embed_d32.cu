@@ -35,7 +35,6 @@ constexpr int kThreads = kWarps * 32;
 struct D32Plan {
     int S;          // states per slice
     int n_slices;
-    int ints_in_smem;
     int x_floats;   // floats of one feature staging buffer (widest level x S x F, padded)
     size_t smem_bytes;
 };
@@ -80,10 +79,9 @@ struct Weights32 {
 template <int R, int KF>
 __device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[KF], int pos,
                                          int q, int s0, bool last_live, int nb, int S, int F,
-                                         int lane, const int *order, const int *nbr_ptr,
-                                         const int *nbr_slot, const int *own_slot, float *msg,
-                                         const float *xs, float *__restrict__ H, size_t B,
-                                         int b_first, float *A, float *Bf) {
+                                         int lane, const int4 *meta, const int *nbr_slot,
+                                         float *msg, const float *xs, float *__restrict__ H,
+                                         size_t B, int b_first, float *A, float *Bf) {
     int st[R];
     float x[R], acc[R];
 #pragma unroll
@@ -92,10 +90,22 @@ __device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[
         x[r] = lane < F ? xs[(q * nb + st[r]) * F + lane] : 0.f;
         acc[r] = 0.f;
     }
-    const int e0 = nbr_ptr[pos], e1 = nbr_ptr[pos + 1];
-    const int slot = own_slot[pos];
-    const int v = order[pos];
-    for (int e = e0; e < e1; ++e) {
+    const int4 m = meta[pos];       // {first neighbour entry, end, own slot, node id}
+    const int e1 = m.y, slot = m.z, v = m.w;
+    int e = m.x;
+    for (; e + 4 <= e1; e += 4) {   // four neighbours at a time: the loads overlap
+        int base[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) base[k] = nbr_slot[e + k] * S;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            float t[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) t[k] = msg[(base[k] + st[r]) * kD + lane];
+            acc[r] += (t[0] + t[1]) + (t[2] + t[3]);
+        }
+    }
+    for (; e < e1; ++e) {
         const int base = nbr_slot[e] * S;
 #pragma unroll
         for (int r = 0; r < R; ++r) acc[r] += msg[(base + st[r]) * kD + lane];
@@ -144,24 +154,21 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     const int nb = min(p.S, B - b_first);
 
     // ---- shared memory: [schedule ints][message slots][feature staging x2][exchange buffers]
-    const int *level_ptr = lv.level_ptr, *order = lv.order, *nbr_ptr = lv.nbr_ptr;
-    const int *nbr_slot = lv.nbr_slot, *own_slot = lv.own_slot;
-    float *fsm = smem;
-    if (p.ints_in_smem) {
-        int *ism = reinterpret_cast<int *>(smem);
-        auto stage = [&](const int *src, int count) {
-            int *dst = ism;
-            for (int i = threadIdx.x; i < count; i += kThreads) dst[i] = src[i];
-            ism += (count + 3) & ~3;
-            return (const int *)dst;
-        };
-        level_ptr = stage(lv.level_ptr, lv.n_levels + 1);
-        order = stage(lv.order, a.n);
-        nbr_ptr = stage(lv.nbr_ptr, a.n + 1);
-        own_slot = stage(lv.own_slot, a.n);
-        nbr_slot = stage(lv.nbr_slot, lv.n_nbr);
-        fsm = reinterpret_cast<float *>(ism);
-    }
+    // one packed record per position: {first neighbour entry, end, own slot, node id}
+    int4 *meta_w = reinterpret_cast<int4 *>(smem);
+    for (int i = threadIdx.x; i < a.n; i += kThreads)
+        meta_w[i] = make_int4(lv.nbr_ptr[i], lv.nbr_ptr[i + 1], lv.own_slot[i], lv.order[i]);
+    const int4 *meta = meta_w;
+    int *ism = reinterpret_cast<int *>(smem) + 4 * a.n;
+    auto stage = [&](const int *src, int count) {
+        int *dst = ism;
+        for (int i = threadIdx.x; i < count; i += kThreads) dst[i] = src[i];
+        ism += (count + 3) & ~3;
+        return (const int *)dst;
+    };
+    const int *level_ptr = stage(lv.level_ptr, lv.n_levels + 1);
+    const int *nbr_slot = stage(lv.nbr_slot, lv.n_nbr);
+    float *fsm = reinterpret_cast<float *>(ism);
     float *msg = fsm;                                       // [n_slots][S][32]
     float *xstage = msg + (size_t)lv.n_slots * p.S * kD;    // [2][x_floats]
     float *xbuf = xstage + 2 * (size_t)p.x_floats + (size_t)warp * 4 * KF;
@@ -186,22 +193,25 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
 
     // Asynchronous copy of one level's raw features (rows of the slice) into a
     // staging buffer, so that the next level's x is on chip when it is needed.
+    // exact division of small non-negative numbers by a per-block constant
+    auto magic_of = [](int d) { return (unsigned)((0x100000000ull + d - 1) / d); };
+    const unsigned magic_nb = magic_of(nb), magic_ppn = magic_of((nb + 1) >> 1);
     const int per_node = nb * F;             // floats per node, contiguous in X
+    const bool vec = (F & 3) == 0;
+    const int per = vec ? per_node >> 2 : per_node;     // copy pieces per node
+    const unsigned magic_per = magic_of(per);
+    // The last warp (the one least often needed for rows) issues all copies, so
+    // the other warps go straight to their rows.
     auto prefetch = [&](int level) {
+        if (warp != kWarps - 1) return;
         const int q0 = level_ptr[level], width = level_ptr[level + 1] - q0;
         float *dst = xstage + (size_t)(level & 1) * p.x_floats;
-        if ((F & 3) == 0) {
-            const int per = per_node >> 2;
-            for (int i = threadIdx.x; i < width * per; i += kThreads) {
-                const int q = i / per, off = (i - q * per) * 4;
-                __pipeline_memcpy_async(dst + q * per_node + off,
-                                        X + ((size_t)order[q0 + q] * B + b_first) * F + off, 16);
-            }
-        } else {
-            for (int i = threadIdx.x; i < width * per_node; i += kThreads) {
-                const int q = i / per_node, off = i - q * per_node;
-                __pipeline_memcpy_async(dst + i, X + ((size_t)order[q0 + q] * B + b_first) * F + off, 4);
-            }
+        for (int i = lane; i < width * per; i += 32) {
+            const int q = per == 1 ? i : (int)__umulhi((unsigned)i, magic_per);
+            const int piece = i - q * per;
+            const float *src = X + ((size_t)meta[q0 + q].w * B + b_first) * F;
+            if (vec) __pipeline_memcpy_async(dst + q * per_node + 4 * piece, src + 4 * piece, 16);
+            else __pipeline_memcpy_async(dst + q * per_node + piece, src + piece, 4);
         }
         __pipeline_commit();
     };
@@ -218,17 +228,19 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         if (rows <= kWarps) {
             // narrow level: one row per warp, shortest dependent chains
             if (warp < rows) {
-                const int q = warp / nb, s0 = warp - q * nb;
-                run_node<1, KF>(w, wf1, p0 + q, q, s0, true, nb, p.S, F, lane, order, nbr_ptr,
-                                nbr_slot, own_slot, msg, xs, H, B, b_first, A, Bf);
+                const int q = nb == 1 ? warp : (int)__umulhi((unsigned)warp, magic_nb);
+                const int s0 = warp - q * nb;
+                run_node<1, KF>(w, wf1, p0 + q, q, s0, true, nb, p.S, F, lane, meta, nbr_slot, msg,
+                                xs, H, B, b_first, A, Bf);
             }
         } else {
             // two states of one node per warp pass
             const int ppn = (nb + 1) >> 1;
             for (int item = warp; item < width * ppn; item += kWarps) {
-                const int q = item / ppn, s0 = (item - q * ppn) * 2;
-                run_node<2, KF>(w, wf1, p0 + q, q, s0, s0 + 1 < nb, nb, p.S, F, lane, order,
-                                nbr_ptr, nbr_slot, own_slot, msg, xs, H, B, b_first, A, Bf);
+                const int q = ppn == 1 ? item : (int)__umulhi((unsigned)item, magic_ppn);
+                const int s0 = (item - q * ppn) * 2;
+                run_node<2, KF>(w, wf1, p0 + q, q, s0, s0 + 1 < nb, nb, p.S, F, lane, meta, nbr_slot,
+                                msg, xs, H, B, b_first, A, Bf);
             }
         }
         __pipeline_wait_prior(0);
@@ -262,29 +274,20 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
     size_t ints = 0;
     for (int dir = 0; dir < 2; ++dir) {
         const DevLevels &lv = a.lv[dir];
-        size_t s = ((lv.n_levels + 1 + 3) & ~3) + 2 * ((a.n + 3) & ~3) + ((a.n + 1 + 3) & ~3) +
-                   ((lv.n_nbr + 3) & ~3);
-        ints = std::max(ints, s);
+        ints = std::max(ints, (size_t)4 * a.n + ((lv.n_levels + 1 + 3) & ~3) + ((lv.n_nbr + 3) & ~3));
     }
     const size_t xbuf = (size_t)kWarps * 4 * KF * sizeof(float);
     auto x_floats = [&](int S) { return (a.max_level_width * S * a.F + 3) & ~3; };
-    auto need = [&](int S, bool with_ints) {
+    auto need = [&](int S) {
         return (size_t)max_slots * S * kD * sizeof(float) + 2 * (size_t)x_floats(S) * sizeof(float) +
-               xbuf + (with_ints ? ints * sizeof(int) : 0);
+               xbuf + ints * sizeof(int);
     };
-    p.ints_in_smem = 1;
-    if (need(p.S, true) > budget) {
-        if (need(p.S, false) <= budget) p.ints_in_smem = 0;
-        else {
-            // narrower slices (more blocks than half the SMs: they queue up)
-            while (p.S > 1 && need(p.S, true) > budget) --p.S;
-            if (need(p.S, true) > budget) p.ints_in_smem = 0;
-            if (need(p.S, p.ints_in_smem != 0) > budget) return cudaErrorNotSupported;
-        }
-    }
+    // narrower slices when the shared memory does not fit (more blocks: they queue up)
+    while (p.S > 1 && need(p.S) > budget) --p.S;
+    if (need(p.S) > budget) return cudaErrorNotSupported;
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.x_floats = x_floats(p.S);
-    p.smem_bytes = need(p.S, p.ints_in_smem != 0);
+    p.smem_bytes = need(p.S);
     void (*kern)(const EmbedArgs, const D32Plan) = nullptr;
     switch (F4) {
         case 1: kern = embed_d32_kernel<1>; break;

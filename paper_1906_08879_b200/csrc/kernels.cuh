@@ -94,6 +94,12 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
 bool embed_d64_applicable(const EmbedArgs &a);
 cudaError_t launch_embed_d64(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
+// embed_mma.cu: d = 32 / 64 on the tensor cores (mma.sync, TF32 operands split
+// into head + tail, three products per step for FP32 accuracy).
+bool embed_mma_applicable(const EmbedArgs &a);
+bool embed_mma_preferred(const EmbedArgs &a);   // applicable and faster than the FMA kernels
+cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
+
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);
 cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);

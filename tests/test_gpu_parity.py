@@ -28,7 +28,8 @@ pytestmark = pytest.mark.gpu
 TOL_ELEM, TOL_NORM = 1e-4, 2e-5
 SCHEDULES = {"sliced": placeto.PLACETO_SLICED, "per_level": placeto.PLACETO_PER_LEVEL,
              "cooperative": placeto.PLACETO_COOPERATIVE,
-             "generic_sliced": placeto.PLACETO_SLICED | placeto.PLACETO_GENERIC}
+             "generic_sliced": placeto.PLACETO_SLICED | placeto.PLACETO_GENERIC,
+             "fma_only": placeto.PLACETO_FMA_ONLY, "tensor": placeto.PLACETO_TENSOR}
 
 
 def dev_t(a):
@@ -115,28 +116,31 @@ def test_inception_normalised():
     compare(cfg, gpu_forward(cfg), oracle.forward(cfg, threads=8))
 
 
+@pytest.mark.parametrize("flags", [0, placeto.PLACETO_TENSOR])
 @pytest.mark.parametrize("normalise", [False, True])
-def test_nmt(normalise):
+def test_nmt(normalise, flags):
     cfg = configs.make("nmt", normalise=normalise)
-    out = gpu_forward(cfg)
+    out = gpu_forward(cfg, flags)
     compare(cfg, out, oracle.forward(cfg, threads=8))
 
 
-def test_nasnet_full_batch_sampled_states():
+@pytest.mark.parametrize("flags", [0, placeto.PLACETO_FMA_ONLY])
+def test_nasnet_full_batch_sampled_states(flags):
     """Full size on the GPU (n ~ 2100, B = 512, d = 64); the checker evaluates
     a sample of states one by one (states are independent)."""
     cfg = configs.make("nasnet")
-    out = gpu_forward(cfg)
+    out = gpu_forward(cfg, flags)
     sel = np.asarray([0, 1, 63, 64, 255, 256, 300, 448, 510, 511])
     compare(cfg, out, oracle.forward(cfg, threads=8, states=sel), sel=sel)
     for k in ("H_down", "H_up", "logits", "probs"):
         assert torch.isfinite(out[k]).all()
 
 
+@pytest.mark.parametrize("flags", [0, placeto.PLACETO_TENSOR])
 @pytest.mark.parametrize("i", [0, 1, 30, 63])
-def test_episode_sweep(i):
+def test_episode_sweep(i, flags):
     cfg = configs.make_sweep(i)
-    out = gpu_forward(cfg)
+    out = gpu_forward(cfg, flags)
     n = cfg["n"]
     sel = None if n <= 320 else np.unique(np.linspace(0, n - 1, 48).astype(int))
     ref = oracle.forward(cfg, threads=8, states=sel)
