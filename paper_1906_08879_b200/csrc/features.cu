@@ -38,19 +38,33 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
     __syncthreads();
     const int nb = min(kTile, B - b0);
     const int nv = min(kTile, n - v0);
-    for (int vl = 0; vl < nv; ++vl) {
+    // one (node, state) pair per thread pass: its F features are contiguous in X,
+    // and the pairs of one node follow each other, so a warp writes 32 F floats in a row
+    for (int i = threadIdx.x; i < nv * kTile; i += blockDim.x) {
+        const int vl = i / kTile, bl = i % kTile;
+        if (bl >= nb) continue;
         const int v = v0 + vl;
-        const float c = s_cost[vl], s = s_bytes[vl];
-        float *out = X + ((size_t)v * B + b0) * F;
-        for (int i = threadIdx.x; i < nb * F; i += blockDim.x) {
-            const int bl = i / F, k = i - bl * F;
-            float val;
-            if (k == 0) val = c;
-            else if (k == 1) val = s;
-            else if (k < 2 + m) val = (s_dev[bl][vl] == k - 2) ? 1.f : 0.f;
-            else if (k == 2 + m) val = (s_cur[bl] == v) ? 1.f : 0.f;
-            else val = s_placed[bl][vl] ? 1.f : 0.f;
-            out[i] = val;
+        float *out = X + ((size_t)v * B + b0 + bl) * F;
+        const int d = s_dev[bl][vl];
+        const float cur_flag = (s_cur[bl] == v) ? 1.f : 0.f;
+        const float placed_flag = s_placed[bl][vl] ? 1.f : 0.f;
+        if ((F & 3) == 0) {
+            for (int k = 0; k < F; k += 4) {
+                float t[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int kk = k + j;
+                    t[j] = kk == 0 ? s_cost[vl] : kk == 1 ? s_bytes[vl]
+                         : kk < 2 + m ? (d == kk - 2 ? 1.f : 0.f)
+                         : kk == 2 + m ? cur_flag : placed_flag;
+                }
+                *reinterpret_cast<float4 *>(out + k) = make_float4(t[0], t[1], t[2], t[3]);
+            }
+        } else {
+            for (int kk = 0; kk < F; ++kk)
+                out[kk] = kk == 0 ? s_cost[vl] : kk == 1 ? s_bytes[vl]
+                        : kk < 2 + m ? (d == kk - 2 ? 1.f : 0.f)
+                        : kk == 2 + m ? cur_flag : placed_flag;
         }
     }
 }

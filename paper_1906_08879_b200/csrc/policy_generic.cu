@@ -9,6 +9,8 @@
 // the set of each node read from the relation row of c). Kernel 2 adds the
 // chunks in a fixed order (deterministic, no atomics), applies h_i, the head and
 // the softmax, eight states per block so that each weight is read once per block.
+#include <cuda_pipeline.h>
+
 #include <algorithm>
 #include <cmath>
 
@@ -130,7 +132,10 @@ pool_partial_kernel(const PoolArgs a, const PoolPlan p) {
 // columns) with eight loads in flight; the parts are then added in a fixed order
 // through `red`. Narrow layers (the device logits): one warp per (row, column),
 // the lanes split the inner dimension and combine with a shuffle reduction.
-__device__ __forceinline__ void head_dense(const float *__restrict__ W,
+// Not inlined on purpose: the kernel calls it eight times and runs each call once,
+// so one shared copy of the code keeps the instruction fetches (cold after an L2
+// flush) to a single pass.
+__device__ __noinline__ void head_dense(const float *__restrict__ W,
                                            const float *__restrict__ bias, int in, int out,
                                            bool relu, const float *src, int src_stride, float *dst,
                                            int dst_stride, float *red) {
@@ -228,8 +233,8 @@ __device__ __forceinline__ void head_mlp(const DevMlp &net, const float *in, int
 }
 
 // One block finishes kHeadStates states: chunk partial sums -> h_i -> head -> softmax.
-__global__ void __launch_bounds__(kHeadThreads)
-pool_head_kernel(const PoolArgs a, int tmp_floats) {
+__global__ void __launch_bounds__(kHeadThreads, 1)
+pool_head_kernel(const PoolArgs a, int tmp_floats, int stage_floats) {
     extern __shared__ __align__(16) float smem[];
     const int d = a.d, F = a.F, B = a.B, m = a.m;
     const int E = 2 * d + F, Z = 5 * d + F;
@@ -240,9 +245,42 @@ pool_head_kernel(const PoolArgs a, int tmp_floats) {
     float *lg = tmp + kHeadStates * tmp_floats;    // [states][m]
     float *red = lg + ((kHeadStates * m + 3) & ~3);   // [blockDim.x * states] partial products
     const int b0 = blockIdx.x * kHeadStates;
-    prefetch_l2(a.head.W1, (size_t)a.head.in_dim * a.head.hidden_dim);
-    if (a.head.n_layers == 2) prefetch_l2(a.head.W2, (size_t)a.head.hidden_dim * a.head.out_dim);
-    for (int i = 0; i < 3; ++i) prefetch_l2(a.h[i].W1, (size_t)a.h[i].in_dim * a.h[i].hidden_dim);
+    // The networks of this kernel: staged whole into shared memory with cp.async
+    // when they fit (one round trip to L2 / DRAM instead of one per layer part),
+    // otherwise read from global memory after an L2 prefetch.
+    DevMlp net_h0 = a.h[0], net_h1 = a.h[1], net_h2 = a.h[2], net_head = a.head;
+    if (stage_floats > 0) {
+        float *w = red + (size_t)blockDim.x * kHeadStates;
+        auto stage = [&](const float *&ptr, size_t count) {
+            if (ptr == nullptr) return;
+            if ((count & 3) == 0) {
+                for (size_t i = (size_t)threadIdx.x * 4; i < count; i += (size_t)blockDim.x * 4)
+                    __pipeline_memcpy_async(w + i, ptr + i, 16);
+            } else {
+                for (size_t i = threadIdx.x; i < count; i += blockDim.x)
+                    __pipeline_memcpy_async(w + i, ptr + i, 4);
+            }
+            ptr = w;
+            w += (count + 3) & ~size_t(3);
+        };
+        auto stage_net = [&](DevMlp &nt) {
+            stage(nt.W1, (size_t)nt.in_dim * nt.hidden_dim);
+            stage(nt.b1, nt.hidden_dim);
+            if (nt.n_layers == 2) {
+                stage(nt.W2, (size_t)nt.hidden_dim * nt.out_dim);
+                stage(nt.b2, nt.out_dim);
+            }
+        };
+        stage_net(net_h0);
+        stage_net(net_h1);
+        stage_net(net_h2);
+        stage_net(net_head);
+        __pipeline_commit();
+    } else {
+        prefetch_l2(a.head.W1, (size_t)a.head.in_dim * a.head.hidden_dim);
+        if (a.head.n_layers == 2) prefetch_l2(a.head.W2, (size_t)a.head.hidden_dim * a.head.out_dim);
+        for (int i = 0; i < 3; ++i) prefetch_l2(a.h[i].W1, (size_t)a.h[i].in_dim * a.h[i].hidden_dim);
+    }
     for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
         const int s = i / (3 * d), j = i - s * 3 * d;
         const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
@@ -261,10 +299,12 @@ pool_head_kernel(const PoolArgs a, int tmp_floats) {
                           : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
         z[s * Zs + k] = v;
     }
+    __pipeline_wait_prior(0);
     __syncthreads();
-    for (int i = 0; i < 3; ++i)
-        head_mlp(a.h[i], sum + i * d, 3 * d, tmp, tmp_floats, z + E + i * d, Zs, red);
-    head_mlp(a.head, z, Zs, tmp, tmp_floats, lg, m, red);
+    head_mlp(net_h0, sum, 3 * d, tmp, tmp_floats, z + E, Zs, red);
+    head_mlp(net_h1, sum + d, 3 * d, tmp, tmp_floats, z + E + d, Zs, red);
+    head_mlp(net_h2, sum + 2 * d, 3 * d, tmp, tmp_floats, z + E + 2 * d, Zs, red);
+    head_mlp(net_head, z, Zs, tmp, tmp_floats, lg, m, red);
     if (threadIdx.x < kHeadStates && b0 + threadIdx.x < B) {
         const int b = b0 + threadIdx.x;
         const float *l = lg + threadIdx.x * m;
@@ -328,15 +368,24 @@ cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
     for (int i = 0; i < 3; ++i)
         if (a.h[i].n_layers == 2) tmp_floats = std::max(tmp_floats, a.h[i].hidden_dim);
     tmp_floats = (tmp_floats + 3) & ~3;
-    const size_t head_smem =
+    size_t head_smem =
         ((size_t)kHeadStates * (((Z + 3) & ~3) + 3 * a.d + tmp_floats + a.m) + 4 +
          (size_t)kHeadThreads * kHeadStates) * sizeof(float);
+    // floats of all networks, each array padded to a multiple of 4
+    size_t stage_floats = 0;
+    for (const DevMlp *nt : {&a.h[0], &a.h[1], &a.h[2], &a.head}) {
+        stage_floats += (((size_t)nt->in_dim * nt->hidden_dim + 3) & ~size_t(3)) + ((nt->hidden_dim + 3) & ~3);
+        if (nt->n_layers == 2)
+            stage_floats += (((size_t)nt->hidden_dim * nt->out_dim + 3) & ~size_t(3)) + ((nt->out_dim + 3) & ~3);
+    }
+    if (head_smem + stage_floats * sizeof(float) <= 200 * 1024) head_smem += stage_floats * sizeof(float);
+    else stage_floats = 0;
     cudaError_t err = cudaFuncSetAttribute(pool_head_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)head_smem);
     if (err != cudaSuccess) return err;
     const int blocks = (a.B + kHeadStates - 1) / kHeadStates;
-    pool_head_kernel<<<blocks, kHeadThreads, head_smem, stream>>>(a, tmp_floats);
+    pool_head_kernel<<<blocks, kHeadThreads, head_smem, stream>>>(a, tmp_floats, (int)stage_floats);
     count_launch();
     return cudaGetLastError();
 }
