@@ -92,6 +92,29 @@ def job_throughput(local_ms: float, states_per_rank: int, steps: int, dist=None,
     return states_per_rank * world * steps / (slowest * 1e-3), slowest
 
 
+def measured_traffic(workload: str):
+    """DRAM bytes per launch of the message-passing kernel from the committed ncu
+    summary of this workload (profiles/*.md), or None when there is none or the
+    kernel source has changed since the counters were taken."""
+    import glob
+    import hashlib
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        fields = {}
+        for line in open(path):
+            if ":" in line and not line.startswith(("|", "#", " ")):
+                k, _, v = line.partition(":")
+                fields[k.strip()] = v.strip()
+        if fields.get("workload") != workload or "traffic_bytes_per_launch" not in fields:
+            continue
+        src = os.path.join(ROOT, fields.get("kernel_source", ""))
+        if not os.path.isfile(src):
+            continue
+        sha = hashlib.sha1(open(src, "rb").read()).hexdigest()[:12]
+        if sha == fields.get("kernel_source_sha1_12"):
+            return int(fields["traffic_bytes_per_launch"]), os.path.basename(path)
+    return None, None
+
+
 # ------------------------------------------------------------ CPU checker ---
 
 def time_oracle(cfg, budget_s: float, threads: int):
@@ -319,9 +342,13 @@ def run_b200(args):
         sm_max_mhz = json.load(open(peaks_path)).get("sm_max_mhz", sm_max_mhz)
     peak_tflops = sm_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
     achieved = flops_embed(cfg) / (embed_ms * 1e-3) / 1e12
+    traffic, traffic_from = measured_traffic(cfg["name"])
     roofline = {"bound": "alu", "kernel": "message passing (embed_forward, %d launch(es))" % embed_launches,
                 "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved / peak_tflops,
-                "traffic": None,
+                "traffic": traffic, "traffic_source": traffic_from,
+                "arithmetic": ("fp32 accumulate on mma.sync, TF32 head+tail operands (3 products)"
+                               if d == 64 and not (args.flags & 16) else "fp32 fma"),
+                "algorithmic_bytes": (4 * F + 8 * d) * n * B,
                 "peak_source": "derived: %d SMs x 128 FP32 FMA lanes x 2 flop x %.0f MHz max SM clock"
                                % (sm_count, sm_max_mhz),
                 "ms_per_launch": embed_ms,
