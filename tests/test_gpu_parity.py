@@ -216,6 +216,26 @@ def test_max_fan_in_node():
     _small_case(n, src, dst, d=32, m=4, B=20, seed=5)
 
 
+@pytest.mark.parametrize("d,m", [(32, 4), (64, 8)])
+def test_very_wide_level_falls_back_to_the_generic_kernel(d, m):
+    """2000 roots -> 40 nodes -> 1 sink: the message slots of one level exceed
+    shared memory, so the specialised kernels decline and the generic one runs."""
+    r = rng(17)
+    roots, mid = 2000, 40
+    src = list(range(roots)) + [roots + i for i in range(mid)]
+    dst = [roots + int(r.integers(0, mid)) for _ in range(roots)] + [roots + mid] * mid
+    _small_case(roots + mid + 1, src, dst, d=d, m=m, B=24, seed=23)
+
+
+@pytest.mark.parametrize("d,m", [(32, 4), (64, 8)])
+def test_long_chain_with_skips(d, m):
+    """Depth 1500: many levels of one node, plus skip edges that keep messages alive."""
+    n = 1500
+    src = list(range(n - 1)) + list(range(0, n - 40, 37))
+    dst = list(range(1, n)) + [i + 40 for i in range(0, n - 40, 37)]
+    _small_case(n, src, dst, d=d, m=m, B=10, seed=29)
+
+
 # ------------------------------------------------------ properties on GPU ---
 
 def test_deterministic_and_batch_independent():
