@@ -129,7 +129,7 @@ def time_oracle(cfg, budget_s: float, threads: int):
         oracle.forward(cfg, threads=threads)
         passes += 1
         el = time.perf_counter() - t0
-        if el >= budget_s or passes >= 50:
+        if el >= budget_s:
             break
     return cfg["B"] * passes / el, el / passes, passes
 
@@ -142,16 +142,20 @@ def run_reference(args):
     cores = len(os.sched_getaffinity(0))
     from oracle import oracle
     oracle.build()
-    steps, warmup = max(1, min(args.steps, 20)), max(1, min(args.warmup, 2))
+    steps, warmup = max(1, args.steps), max(1, args.warmup)
     sample = cfg
-    # bound the work per step to roughly a second
-    est = 1e-9 * (flops_embed(cfg) + flops_pool(cfg)) / max(cores, 1) * 2.0
-    sample_desc = "full batch of %d states per step" % cfg["B"]
-    states_sel = None
-    if est > 2.0:
-        keep = max(cores, int(cfg["B"] * 2.0 / est))
-        states_sel = np.arange(min(keep, cfg["B"]))
-        sample_desc = "first %d of %d states per step" % (len(states_sel), cfg["B"])
+    # Bound the sample of states per step so that the whole run stays near two
+    # minutes: time a probe of one state per core, then size the sample.
+    probe = np.arange(min(cfg["B"], cores))
+    oracle.forward(cfg, threads=cores, states=probe)
+    t0 = time.perf_counter()
+    oracle.forward(cfg, threads=cores, states=probe)
+    per_state = (time.perf_counter() - t0) / len(probe)
+    keep = int(120.0 / (steps + warmup) / max(per_state, 1e-9))
+    keep = max(min(cores, cfg["B"]), min(cfg["B"], keep))
+    states_sel = None if keep >= cfg["B"] else np.arange(keep)
+    sample_desc = ("full batch of %d states per step" % cfg["B"] if states_sel is None
+                   else "first %d of %d states per step" % (keep, cfg["B"]))
     nstates = cfg["B"] if states_sel is None else len(states_sel)
     for _ in range(warmup):
         oracle.forward(sample, threads=cores, states=states_sel)
