@@ -45,11 +45,11 @@ struct D32Plan {
 template <int R, int K>
 __device__ __forceinline__ void matvec(const float (&w)[K], float bias, const float *in,
                                        int row_stride, float (&out)[R]) {
-    float acc[R][4];
+    float acc[R][2];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         acc[r][0] = bias;
-        acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+        acc[r][1] = 0.f;
     }
 #pragma unroll
     for (int k = 0; k < K; k += 4) {
@@ -58,12 +58,12 @@ __device__ __forceinline__ void matvec(const float (&w)[K], float bias, const fl
             const float4 u = *reinterpret_cast<const float4 *>(in + r * row_stride + k);
             acc[r][0] = fmaf(u.x, w[k], acc[r][0]);
             acc[r][1] = fmaf(u.y, w[k + 1], acc[r][1]);
-            acc[r][2] = fmaf(u.z, w[k + 2], acc[r][2]);
-            acc[r][3] = fmaf(u.w, w[k + 3], acc[r][3]);
+            acc[r][0] = fmaf(u.z, w[k + 2], acc[r][0]);
+            acc[r][1] = fmaf(u.w, w[k + 3], acc[r][1]);
         }
     }
 #pragma unroll
-    for (int r = 0; r < R; ++r) out[r] = (acc[r][0] + acc[r][1]) + (acc[r][2] + acc[r][3]);
+    for (int r = 0; r < R; ++r) out[r] = acc[r][0] + acc[r][1];
 }
 
 struct Weights32 {
