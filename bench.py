@@ -344,6 +344,10 @@ def run_b200(args):
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
         sm_max_mhz = json.load(open(peaks_path)).get("sm_max_mhz", sm_max_mhz)
+    hbm_peak, hbm_src = 6650.0, "fallback (earlier measurement on this pool)"
+    if os.path.exists(peaks_path):
+        hbm_peak = float(json.load(open(peaks_path)).get("hbm_gbs", hbm_peak))
+        hbm_src = "measured (MEASURED_PEAKS.json)"
     peak_tflops = sm_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
     achieved = flops_embed(cfg) / (embed_ms * 1e-3) / 1e12
     traffic, traffic_from = measured_traffic(cfg["name"])
@@ -353,6 +357,9 @@ def run_b200(args):
                 "arithmetic": ("fp32 accumulate on mma.sync, TF32 head+tail operands (3 products)"
                                if d == 64 and not (args.flags & 16) else "fp32 fma"),
                 "algorithmic_bytes": (4 * F + 8 * d) * n * B,
+                "hbm": {"achieved": (4 * F + 8 * d) * n * B / (embed_ms * 1e-3) / 1e9, "peak": hbm_peak,
+                        "unit": "GB/s", "frac": (4 * F + 8 * d) * n * B / (embed_ms * 1e-3) / 1e9 / hbm_peak,
+                        "peak_source": hbm_src},
                 "peak_source": "derived: %d SMs x 128 FP32 FMA lanes x 2 flop x %.0f MHz max SM clock"
                                % (sm_count, sm_max_mhz),
                 "ms_per_launch": embed_ms,
