@@ -284,8 +284,17 @@ pool_head_kernel(const PoolArgs a, int tmp_floats, int stage_floats) {
     for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
         const int s = i / (3 * d), j = i - s * 3 * d;
         const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
+        // chunks are added in ascending order; four loads in flight at a time
+        const float *src = a.partial + (size_t)b * 3 * d + j;
+        const size_t step = (size_t)B * 3 * d;
         float acc = 0.f;
-        for (int ch = 0; ch < a.chunks; ++ch) acc += a.partial[((size_t)ch * B + b) * 3 * d + j];
+        int ch = 0;
+        for (; ch + 4 <= a.chunks; ch += 4) {
+            const float t0 = src[ch * step], t1 = src[(ch + 1) * step];
+            const float t2 = src[(ch + 2) * step], t3 = src[(ch + 3) * step];
+            acc = (((acc + t0) + t1) + t2) + t3;
+        }
+        for (; ch < a.chunks; ++ch) acc += src[ch * step];
         sum[i] = acc;
     }
     for (int i = threadIdx.x; i < kHeadStates * E; i += blockDim.x) {
@@ -301,9 +310,29 @@ pool_head_kernel(const PoolArgs a, int tmp_floats, int stage_floats) {
     }
     __pipeline_wait_prior(0);
     __syncthreads();
-    head_mlp(net_h0, sum, 3 * d, tmp, tmp_floats, z + E, Zs, red);
-    head_mlp(net_h1, sum + d, 3 * d, tmp, tmp_floats, z + E + d, Zs, red);
-    head_mlp(net_h2, sum + 2 * d, 3 * d, tmp, tmp_floats, z + E + 2 * d, Zs, red);
+    if (net_h0.n_layers == 1 && net_h1.n_layers == 1 && net_h2.n_layers == 1) {
+        // the three single-layer h_i in one pass: thread = (row, set, column)
+        for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
+            const int s = i / (3 * d), r = i - s * 3 * d;
+            const int set = r / d, j = r - set * d;
+            const DevMlp &nt = set == 0 ? net_h0 : (set == 1 ? net_h1 : net_h2);
+            const float *v = sum + s * 3 * d + set * d;
+            float a0 = nt.b1[j], a1 = 0.f;
+            int k = 0;
+            for (; k + 2 <= d; k += 2) {
+                a0 = fmaf(v[k], nt.W1[(size_t)k * d + j], a0);
+                a1 = fmaf(v[k + 1], nt.W1[(size_t)(k + 1) * d + j], a1);
+            }
+            if (k < d) a0 = fmaf(v[k], nt.W1[(size_t)k * d + j], a0);
+            const float y = a0 + a1;
+            z[s * Zs + E + r] = (nt.act == 0 && nt.final_act) ? fmaxf(y, 0.f) : y;
+        }
+        __syncthreads();
+    } else {
+        head_mlp(net_h0, sum, 3 * d, tmp, tmp_floats, z + E, Zs, red);
+        head_mlp(net_h1, sum + d, 3 * d, tmp, tmp_floats, z + E + d, Zs, red);
+        head_mlp(net_h2, sum + 2 * d, 3 * d, tmp, tmp_floats, z + E + 2 * d, Zs, red);
+    }
     head_mlp(net_head, z, Zs, tmp, tmp_floats, lg, m, red);
     if (threadIdx.x < kHeadStates && b0 + threadIdx.x < B) {
         const int b = b0 + threadIdx.x;
