@@ -188,6 +188,20 @@ def test_widths(d, m):
     _small_case(24, src, dst, d=d, m=m, B=9, seed=d)
 
 
+@pytest.mark.parametrize("d", [32, 64])
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 8, 11, 12])
+def test_specialised_kernels_over_feature_widths(d, m):
+    """F = m + 4 from 5 to 16: vector and scalar feature prefetch, every padded
+    first-layer width of the d = 32 / 64 kernels, pooling with and without the
+    fast path (it needs F to be a multiple of 4)."""
+    r = rng(100 * d + m)
+    n = int(r.integers(30, 90))
+    src, dst = random_dag(r, n, float(r.uniform(0.03, 0.12)))
+    B = int(r.integers(3, 70))
+    for flags in (0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR):
+        _small_case(n, src, dst, d=d, m=m, B=B, seed=m + d, schedule=flags)
+
+
 def test_single_layer_networks_as_in_the_paper():
     """Appendix A.7: single-layer f, g (hidden = input width)."""
     r = rng(9)
