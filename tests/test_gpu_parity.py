@@ -314,6 +314,27 @@ def test_policy_forward_and_host_variant_match_the_separate_calls():
     assert torch.equal(h_logits, ref["logits"].cpu()) and torch.equal(h_probs, ref["probs"].cpu())
 
 
+def test_two_streams_with_their_own_workspaces_do_not_interfere():
+    cfg = configs.make("inception")
+    ref = gpu_forward(cfg)
+    g, w = ref["graph"], ref["w"]
+    B, m = cfg["B"], cfg["m"]
+    ins = [dev_t(cfg[k]) for k in ("cost", "bytes", "dev", "cur", "placed")]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    torch.cuda.synchronize()
+    for st in streams:
+        ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD)
+        logits = torch.empty((B, m), device="cuda")
+        probs = torch.empty((B, m), device="cuda")
+        for _ in range(3):
+            placeto.placeto_policy_forward(g, w, *ins, logits, probs, ws, 0, st)
+        outs.append((logits, probs, ws))
+    torch.cuda.synchronize()
+    for logits, probs, _ in outs:
+        assert torch.equal(logits, ref["logits"]) and torch.equal(probs, ref["probs"])
+
+
 # ---------------------------------------------------------- error handling ---
 
 def test_argument_errors_are_reported_not_faulted():

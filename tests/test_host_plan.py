@@ -136,6 +136,21 @@ def test_plan_rejects_bad_graphs():
     assert status(1 << 20, [], []) == 1                # beyond the node limit
 
 
+def test_plan_at_the_node_limit():
+    n = 16384                                           # PLACETO_MAX_NODES
+    src = np.arange(n - 1, dtype=np.int32)
+    g = placeto.Graph(n, src, src + 1, host_only=True)  # a chain: depth n, two alternating slots
+    info = g.info()
+    assert info["n_levels_down"] == n and info["max_level_width"] == 1
+    view = g.host_view()
+    assert view["down"]["n_slots"] == 2 and view["up"]["n_slots"] == 2
+    rel = view["relation"]
+    assert rel[0, n - 1] == 1 and rel[n - 1, 0] == 0 and rel[5, 5] == 3
+    g.close()
+    with pytest.raises(placeto.PlacetoError):
+        placeto.Graph(n + 1, src, src + 1, host_only=True)
+
+
 def test_workspace_bytes_on_host_graph():
     cfg = configs.make("tiny")
     g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"], host_only=True)
