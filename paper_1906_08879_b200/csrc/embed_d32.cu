@@ -93,6 +93,15 @@ __device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[
     const int4 m = meta[pos];       // {first neighbour entry, end, own slot, node id}
     const int e1 = m.y, slot = m.z, v = m.w;
     int e = m.x;
+    if (e1 - e == 1) {
+        // One neighbour (most nodes of chain-like graphs): its message row is the
+        // input of g as it stands, so the first layer reads the slot directly and
+        // the gather, the store and the warp barrier are skipped.
+        const float *row = msg + (nbr_slot[e] * S + st[0]) * kD;
+        matvec<R, kD>(w.g1, w.bg1, row, (R > 1 && last_live) ? kD : 0, acc);
+        __syncwarp();               // the previous node's last reads of Bf are done
+        goto after_g1;
+    }
     for (; e + 4 <= e1; e += 4) {   // four neighbours at a time: the loads overlap
         int base[4];
 #pragma unroll
@@ -114,6 +123,7 @@ __device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[
     for (int r = 0; r < R; ++r) A[r * KF + lane] = acc[r];
     __syncwarp();
     matvec<R, kD>(w.g1, w.bg1, A, KF, acc);
+after_g1:
 #pragma unroll
     for (int r = 0; r < R; ++r) Bf[r * KF + lane] = fmaxf(acc[r], 0.f);
     __syncwarp();
