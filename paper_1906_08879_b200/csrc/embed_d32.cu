@@ -90,14 +90,15 @@ __device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[
         x[r] = lane < F ? xs[(q * nb + st[r]) * F + lane] : 0.f;
         acc[r] = 0.f;
     }
-    const int4 m = meta[pos];       // {first neighbour entry, end, own slot, node id}
-    const int e1 = m.y, slot = m.z, v = m.w;
+    const int4 m = meta[pos];       // {first neighbour entry, end, own | first neighbour slot, node}
+    const int e1 = m.y, v = m.w;
+    const int slot = (m.z & 0xffff) == 0xffff ? -1 : (m.z & 0xffff);
     int e = m.x;
     if (e1 - e == 1) {
         // One neighbour (most nodes of chain-like graphs): its message row is the
         // input of g as it stands, so the first layer reads the slot directly and
         // the gather, the store and the warp barrier are skipped.
-        const float *row = msg + (nbr_slot[e] * S + st[0]) * kD;
+        const float *row = msg + ((int)((unsigned)m.z >> 16) * S + st[0]) * kD;
         matvec<R, kD>(w.g1, w.bg1, row, (R > 1 && last_live) ? kD : 0, acc);
         __syncwarp();               // the previous node's last reads of Bf are done
         goto after_g1;
@@ -164,10 +165,14 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     const int nb = min(p.S, B - b_first);
 
     // ---- shared memory: [schedule ints][message slots][feature staging x2][exchange buffers]
-    // one packed record per position: {first neighbour entry, end, own slot, node id}
+    // one packed record per position: {first neighbour entry, end,
+    // own slot (low 16 bits, 0xffff = none) | slot of the first neighbour (high 16 bits), node id}
     int4 *meta_w = reinterpret_cast<int4 *>(smem);
-    for (int i = threadIdx.x; i < a.n; i += kThreads)
-        meta_w[i] = make_int4(lv.nbr_ptr[i], lv.nbr_ptr[i + 1], lv.own_slot[i], lv.order[i]);
+    for (int i = threadIdx.x; i < a.n; i += kThreads) {
+        const int e0 = lv.nbr_ptr[i], e1 = lv.nbr_ptr[i + 1];
+        const int first = e1 > e0 ? lv.nbr_slot[e0] : 0;
+        meta_w[i] = make_int4(e0, e1, (lv.own_slot[i] & 0xffff) | (first << 16), lv.order[i]);
+    }
     const int4 *meta = meta_w;
     int *ism = reinterpret_cast<int *>(smem) + 4 * a.n;
     auto stage = [&](const int *src, int count) {
@@ -281,6 +286,7 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
     const int KF = kD + 4 * F4;
     const size_t budget = (size_t)std::min(di.max_smem_optin, 227 * 1024) - 1024;
     const int max_slots = std::max(a.lv[0].n_slots, a.lv[1].n_slots);
+    if (max_slots >= 0xffff) return cudaErrorNotSupported;   // slot ids are packed into 16 bits
     size_t ints = 0;
     for (int dir = 0; dir < 2; ++dir) {
         const DevLevels &lv = a.lv[dir];
