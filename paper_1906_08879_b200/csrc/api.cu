@@ -138,7 +138,7 @@ placeto_status cuda_status(cudaError_t e) {
 
 placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const float *X, int B,
                          float *H_down, float *H_up, char *ws, const Layout &L, uint32_t flags,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, bool after_own_kernel = false) {
     EmbedArgs a;
     a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
     a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
@@ -152,11 +152,11 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     const unsigned schedule = pick_schedule(flags);
     const bool want_mma = (flags & PLACETO_TENSOR) ? embed_mma_applicable(a) : embed_mma_preferred(a);
     if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) && schedule == PLACETO_SLICED && want_mma) {
-        cudaError_t e = launch_embed_mma(a, g->info, stream);
+        cudaError_t e = launch_embed_mma(a, g->info, stream, after_own_kernel);
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
     if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d32_applicable(a)) {
-        cudaError_t e = launch_embed_d32(a, g->info, stream);
+        cudaError_t e = launch_embed_d32(a, g->info, stream, after_own_kernel);
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
     if (!(flags & PLACETO_GENERIC) && schedule == PLACETO_SLICED && embed_d64_applicable(a)) {
@@ -169,7 +169,7 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
 placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const float *X,
                         const float *H_down, const float *H_up, const int32_t *cur, int B,
                         float *logits, float *probs, char *ws, const Layout &L, uint32_t flags,
-                        cudaStream_t stream) {
+                        cudaStream_t stream, bool after_own_kernel = false) {
     PoolArgs a;
     for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
     a.head = to_dev(w->head);
@@ -182,7 +182,8 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     const bool fast32 = pool_d32_applicable(a), fast64 = pool_d64_applicable(a);
     if (!(flags & PLACETO_GENERIC) && L.chunks32 > 0 && (fast32 || fast64)) {
         a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
-        cudaError_t e = fast32 ? launch_pool_d32(a, g->info, stream) : launch_pool_d64(a, g->info, stream);
+        cudaError_t e = fast32 ? launch_pool_d32(a, g->info, stream, after_own_kernel)
+                               : launch_pool_d64(a, g->info, stream, after_own_kernel);
         if (e == cudaSuccess) return cuda_status(launch_pool_head(a, stream));
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
@@ -449,9 +450,9 @@ placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weig
     float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
     s = cuda_status(launch_features(g->host.n, B, w->m, cost, bytes, dev, cur, placed, X, st));
     if (s != PLACETO_OK) return s;
-    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st);
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;
-    return run_pool(g, w, X, Hd, Hu, cur, B, logits, probs, ws, L, flags, st);
+    return run_pool(g, w, X, Hd, Hu, cur, B, logits, probs, ws, L, flags, st, true);
 }
 
 placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto_weights *w,
@@ -492,9 +493,9 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
     s = cuda_status(launch_features(g->host.n, B, w->m, d_cost, d_bytes, d_dev, d_cur, d_placed, X, st));
     if (s != PLACETO_OK) return s;
-    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st);
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;
-    s = run_pool(g, w, X, Hd, Hu, d_cur, B, d_logits, probs ? d_probs : nullptr, ws, L, flags, st);
+    s = run_pool(g, w, X, Hd, Hu, d_cur, B, d_logits, probs ? d_probs : nullptr, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;
     if (cudaMemcpyAsync(logits, d_logits, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return PLACETO_ERR_CUDA;

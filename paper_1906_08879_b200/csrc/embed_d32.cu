@@ -157,6 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     constexpr int KF = kD + 4 * F4;      // padded input width of f's first layer
     extern __shared__ __align__(16) float smem[];
+    dependents_may_start();
     const int dir = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const DevLevels lv = a.lv[dir];
@@ -230,6 +231,7 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         }
         __pipeline_commit();
     };
+    dependency_wait();          // the raw features may come from a kernel that is still running
     prefetch(0);
     __pipeline_wait_prior(0);
     __syncthreads();
@@ -277,7 +279,8 @@ bool embed_d32_applicable(const EmbedArgs &a) {
     return true;
 }
 
-cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                             bool overlap) {
     D32Plan p;
     const int target = std::max(1, di.sm_count / 2);            // blocks per direction
     const int want = std::max(1, std::min(a.B, target));
@@ -315,9 +318,9 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)p.smem_bytes);
     if (err != cudaSuccess) return err;
-    kern<<<dim3(p.n_slices, 2), kThreads, p.smem_bytes, stream>>>(a, p);
+    err = launch_overlapped(overlap, kern, dim3(p.n_slices, 2), dim3(kThreads), p.smem_bytes, stream, a, p);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace placeto

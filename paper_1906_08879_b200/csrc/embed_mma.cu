@@ -142,6 +142,7 @@ embed_mma_kernel(const EmbedArgs a, const MmaPlan p) {
     constexpr int P = KF + 4;                       // exchange row stride (P mod 8 == 4)
     constexpr int NKD = D / 8;
     extern __shared__ __align__(16) float smem[];
+    dependents_may_start();
     const int group = threadIdx.x / GT;             // d = 32: 0 top-down, 1 bottom-up
     const int dir = D == 32 ? group : (int)blockIdx.y;
     const int gt = threadIdx.x - group * GT;
@@ -216,6 +217,7 @@ embed_mma_kernel(const EmbedArgs a, const MmaPlan p) {
         __pipeline_commit();
     };
     group_sync();                 // schedule staged
+    dependency_wait();            // the raw features may come from a kernel that is still running
     prefetch(0);
     __pipeline_wait_prior(0);
     group_sync();
@@ -327,7 +329,7 @@ bool relu2(const DevMlp &m, int in) {
 }
 
 template <int D, int NKF>
-cudaError_t launch(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+cudaError_t launch(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap) {
     constexpr int P = 8 * NKF + 4;
     MmaPlan p;
     const int dirs_per_block = D == 32 ? 2 : 1;
@@ -361,9 +363,9 @@ cudaError_t launch(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)p.smem_bytes);
     if (err != cudaSuccess) return err;
-    kern<<<dim3(p.n_slices, D == 32 ? 1 : 2), 256, p.smem_bytes, stream>>>(a, p);
+    err = launch_overlapped(overlap, kern, dim3(p.n_slices, D == 32 ? 1 : 2), dim3(256), p.smem_bytes, stream, a, p);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace
@@ -382,10 +384,11 @@ bool embed_mma_applicable(const EmbedArgs &a) {
 // than one 16-row tile and the long MMA latency sits on the level-to-level path.
 bool embed_mma_preferred(const EmbedArgs &a) { return embed_mma_applicable(a) && a.d == 64; }
 
-cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                             bool overlap) {
     const int f8 = (a.F + 7) / 8;      // 1 or 2
-    if (a.d == 32) return f8 == 1 ? launch<32, 5>(a, di, stream) : launch<32, 6>(a, di, stream);
-    if (a.d == 64) return f8 == 1 ? launch<64, 9>(a, di, stream) : launch<64, 10>(a, di, stream);
+    if (a.d == 32) return f8 == 1 ? launch<32, 5>(a, di, stream, overlap) : launch<32, 6>(a, di, stream, overlap);
+    if (a.d == 64) return f8 == 1 ? launch<64, 9>(a, di, stream, overlap) : launch<64, 10>(a, di, stream, overlap);
     return cudaErrorNotSupported;
 }
 

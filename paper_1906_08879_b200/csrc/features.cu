@@ -17,6 +17,7 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
                 const float *__restrict__ bytes, const uint8_t *__restrict__ dev,
                 const int *__restrict__ cur, const uint8_t *__restrict__ placed,
                 float *__restrict__ X) {
+    dependents_may_start();
     __shared__ uint8_t s_dev[kTile][kTile + 4];
     __shared__ uint8_t s_placed[kTile][kTile + 4];
     __shared__ int s_cur[kTile];

@@ -73,6 +73,36 @@ struct DeviceInfo {
 // Counts launches of the calling thread's current forward call.
 void count_launch(int k = 1);
 
+// Programmatic dependent launch. Inside one forward call the library's kernels
+// follow each other on the stream; a kernel launched with launch_overlapped may
+// start while its predecessor is still running and do the part of its set-up
+// that reads nothing the predecessor writes (schedule staging, weights), then
+// calls dependency_wait() before it touches the predecessor's output. The
+// predecessor allows this with dependents_may_start(). Only launches whose
+// predecessor is a kernel of this library use it: weights and other caller
+// inputs may have been written by the caller's own previous kernel, which the
+// first launch of every call waits for in the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dependents_may_start() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 // features.cu
 cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
@@ -87,7 +117,8 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
 // networks of hidden width 32; returns cudaErrorNotSupported when the shapes or
 // the shared-memory budget do not fit (the caller then uses the generic kernel).
 bool embed_d32_applicable(const EmbedArgs &a);
-cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
+cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                             bool overlap = false);
 
 // embed_d64.cu: the same for d = 64 (four-warp column-split groups, both
 // directions in one block).
@@ -98,7 +129,8 @@ cudaError_t launch_embed_d64(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
 // into head + tail, three products per step for FP32 accuracy).
 bool embed_mma_applicable(const EmbedArgs &a);
 bool embed_mma_preferred(const EmbedArgs &a);   // applicable and faster than the FMA kernels
-cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream);
+cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                             bool overlap = false);
 
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);
@@ -109,11 +141,13 @@ cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream);
 // policy_d32.cu: specialised partial sums for d = 32, F a multiple of 4, single-layer ReLU l_i
 bool pool_d32_applicable(const PoolArgs &a);
 void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
-cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
+cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                            bool overlap = false);
 
 // policy_d64.cu: the same for d = 64 (weights of all three sets split over the block's warps)
 bool pool_d64_applicable(const PoolArgs &a);
 void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
-cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
+cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                            bool overlap = false);
 
 }  // namespace placeto

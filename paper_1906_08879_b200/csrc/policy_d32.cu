@@ -52,6 +52,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     constexpr int FP = 4 * F4;             // padded feature width
     constexpr int E = 2 * kD + FP;
     extern __shared__ __align__(16) float smem[];
+    dependents_may_start();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n = a.n, B = a.B, F = a.F;
     const int chunk = blockIdx.x;
@@ -74,6 +75,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
         }
         if (threadIdx.x < kD) bs[i * kD + threadIdx.x] = a.l[i].b1[threadIdx.x];
     }
+    dependency_wait();          // the embeddings may come from a kernel that is still running
     {
         const int per_h = nb * kD / 4;                  // 16-byte pieces per node
         for (int t = threadIdx.x; t < nu * per_h; t += kThreads) {
@@ -170,7 +172,8 @@ void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes
     *chunks = (n + *chunk_nodes - 1) / *chunk_nodes;
 }
 
-cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                            bool overlap) {
     Pool32Plan p;
     p.chunk_nodes = a.chunk_nodes;
     p.chunks = a.chunks;
@@ -189,9 +192,9 @@ cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_
                                            (int)p.smem_bytes);
     if (err != cudaSuccess) return err;
     dim3 grid(p.chunks, (a.B + kWarps - 1) / kWarps);
-    kern<<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
+    err = launch_overlapped(overlap, kern, grid, dim3(kThreads), p.smem_bytes, stream, a, p);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace placeto

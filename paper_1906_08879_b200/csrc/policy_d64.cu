@@ -89,6 +89,8 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     constexpr int KQ = ((E + 3) / 4 + 3) & ~3;      // inner width per lane quarter
     constexpr int RS = 4 * KQ;                      // shared row stride (>= E, zero padded)
     extern __shared__ __align__(16) float smem[];
+    dependents_may_start();
+    dependency_wait();          // the embeddings may come from a kernel that is still running
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int quarter = lane >> 3, col = warp * 8 + (lane & 7);
     const int n = a.n, B = a.B, F = a.F;
@@ -200,7 +202,8 @@ void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes
     *chunks = (n + *chunk_nodes - 1) / *chunk_nodes;
 }
 
-cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                            bool overlap) {
     Pool64Plan p;
     p.chunk_nodes = a.chunk_nodes;
     p.chunks = a.chunks;
@@ -219,9 +222,9 @@ cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_
                                            (int)p.smem_bytes);
     if (err != cudaSuccess) return err;
     dim3 grid(p.chunks, (a.B + kTileStates - 1) / kTileStates);
-    kern<<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
+    err = launch_overlapped(overlap, kern, grid, dim3(kThreads), p.smem_bytes, stream, a, p);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace placeto

@@ -36,6 +36,7 @@ struct PoolPlan {
 __global__ void __launch_bounds__(kPoolThreads)
 pool_partial_kernel(const PoolArgs a, const PoolPlan p) {
     extern __shared__ __align__(16) float smem[];
+    dependents_may_start();
     const int d = a.d, F = a.F, n = a.n, B = a.B;
     const int E = 2 * d + F;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -281,6 +282,7 @@ pool_head_kernel(const PoolArgs a, int tmp_floats, int stage_floats) {
         if (a.head.n_layers == 2) prefetch_l2(a.head.W2, (size_t)a.head.hidden_dim * a.head.out_dim);
         for (int i = 0; i < 3; ++i) prefetch_l2(a.h[i].W1, (size_t)a.h[i].in_dim * a.h[i].hidden_dim);
     }
+    dependency_wait();          // the partial sums come from a kernel that may still be running
     for (int i = threadIdx.x; i < kHeadStates * 3 * d; i += blockDim.x) {
         const int s = i / (3 * d), j = i - s * 3 * d;
         const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
@@ -414,9 +416,11 @@ cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
                                            (int)head_smem);
     if (err != cudaSuccess) return err;
     const int blocks = (a.B + kHeadStates - 1) / kHeadStates;
-    pool_head_kernel<<<blocks, kHeadThreads, head_smem, stream>>>(a, tmp_floats, (int)stage_floats);
+    // always preceded by one of this library's pooling kernels on the same stream
+    err = launch_overlapped(true, pool_head_kernel, dim3(blocks), dim3(kHeadThreads), head_smem, stream, a,
+                            tmp_floats, (int)stage_floats);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace placeto
