@@ -184,7 +184,7 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
         a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
         cudaError_t e = fast32 ? launch_pool_d32(a, g->info, stream, after_own_kernel)
                                : launch_pool_d64(a, g->info, stream, after_own_kernel);
-        if (e == cudaSuccess) return cuda_status(launch_pool_head(a, stream));
+        if (e == cudaSuccess) return cuda_status(launch_pool_head(a, g->info, stream));
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
     a.chunks = L.chunks; a.chunk_nodes = L.chunk_nodes;

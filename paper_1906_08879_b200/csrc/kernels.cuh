@@ -136,7 +136,7 @@ cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
 int pool_chunks(int n, int B, const DeviceInfo &di);
 cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
 // adds the chunk partial sums, applies h_i, the head and the softmax (one block per state)
-cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream);
+cudaError_t launch_pool_head(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
 
 // policy_d32.cu: specialised partial sums for d = 32, F a multiple of 4, single-layer ReLU l_i
 bool pool_d32_applicable(const PoolArgs &a);

@@ -353,6 +353,193 @@ pool_head_kernel(const PoolArgs a, int tmp_floats, int stage_floats) {
     }
 }
 
+// The same finish for the common shapes (single-layer h_i of width d, two-layer
+// head whose hidden width is a multiple of 4) with HS states per block, HS chosen
+// so that the blocks cover the device: a small batch is spread over many SMs
+// instead of eight states sharing one. Nothing is staged: weights are read once
+// per block straight from L2 as 128-bit loads, a thread of the first head layer
+// owns a (states x 4 columns) register tile and one part of the inner dimension,
+// and activations sit transposed in shared memory ([k][state]) so that a tile's
+// states come with one broadcast load. Parts are added in a fixed order.
+constexpr int kFastThreads = 512;
+
+template <int HS>
+__global__ void __launch_bounds__(kFastThreads, 1)
+pool_head_fast_kernel(const PoolArgs a) {
+    constexpr int SR = HS < 4 ? HS : 4;     // states of a thread tile
+    constexpr int SG = HS / SR;             // state groups
+    extern __shared__ __align__(16) float smem[];
+    const int d = a.d, F = a.F, B = a.B, m = a.m;
+    const int E = 2 * d + F, Z = 5 * d + F, Hd = a.head.hidden_dim;
+    float *zt = smem;                              // [Z][HS]: e_c, then the three h_i outputs
+    float *sum = zt + Z * HS;                      // [HS][3 d]
+    float *hid = sum + HS * 3 * d;                 // [Hd][HS]
+    float *lg = hid + Hd * HS;                     // [HS][m]
+    float *red = lg + ((HS * m + 3) & ~3);         // [parts][Hd][HS]
+    const int b0 = blockIdx.x * HS;
+    prefetch_l2(a.head.W1, (size_t)Z * Hd);
+    prefetch_l2(a.head.W2, (size_t)Hd * m);
+    for (int i = 0; i < 3; ++i) prefetch_l2(a.h[i].W1, (size_t)d * d);
+    dependency_wait();          // the partial sums come from a kernel that may still be running
+    for (int i = threadIdx.x; i < HS * 3 * d; i += blockDim.x) {
+        const int s = i / (3 * d), j = i - s * 3 * d;
+        const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
+        // chunks are added in ascending order; four loads in flight at a time
+        const float *src = a.partial + (size_t)b * 3 * d + j;
+        const size_t step = (size_t)B * 3 * d;
+        float acc = 0.f;
+        int ch = 0;
+        for (; ch + 4 <= a.chunks; ch += 4) {
+            const float t0 = src[ch * step], t1 = src[(ch + 1) * step];
+            const float t2 = src[(ch + 2) * step], t3 = src[(ch + 3) * step];
+            acc = (((acc + t0) + t1) + t2) + t3;
+        }
+        for (; ch < a.chunks; ++ch) acc += src[ch * step];
+        sum[i] = acc;
+    }
+    for (int i = threadIdx.x; i < HS * E; i += blockDim.x) {
+        const int s = i / E, k = i - s * E;
+        const int b = min(b0 + s, B - 1);
+        const int c = a.cur[b];
+        float v = 0.f;
+        if (c >= 0 && c < a.n)
+            v = k < d ? a.H[0][((size_t)c * B + b) * d + k]
+              : k < 2 * d ? a.H[1][((size_t)c * B + b) * d + (k - d)]
+                          : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
+        zt[k * HS + s] = v;
+    }
+    __syncthreads();
+    // the three h_i: thread = (state, set, four columns)
+    const int dq = d >> 2;
+    for (int i = threadIdx.x; i < HS * 3 * dq; i += blockDim.x) {
+        const int s = i / (3 * dq), r = i - s * 3 * dq;
+        const int set = r / dq, cq = r - set * dq;
+        const DevMlp &nt = a.h[set];
+        const float *__restrict__ W = nt.W1 + 4 * cq;
+        const float *v = sum + s * 3 * d + set * d;
+        float4 acc = *reinterpret_cast<const float4 *>(nt.b1 + 4 * cq);
+#pragma unroll 8
+        for (int k = 0; k < d; ++k) {
+            const float4 w = __ldg(reinterpret_cast<const float4 *>(W + (size_t)k * d));
+            const float x = v[k];
+            acc.x = fmaf(x, w.x, acc.x); acc.y = fmaf(x, w.y, acc.y);
+            acc.z = fmaf(x, w.z, acc.z); acc.w = fmaf(x, w.w, acc.w);
+        }
+        if (nt.act == 0 && nt.final_act) {
+            acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f);
+            acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f);
+        }
+        float *o = zt + (E + set * d + 4 * cq) * HS + s;
+        o[0] = acc.x; o[HS] = acc.y; o[2 * HS] = acc.z; o[3 * HS] = acc.w;
+    }
+    __syncthreads();
+    // head, first layer
+    const int CG = Hd >> 2, tiles = SG * CG;
+    const int parts = max(1, min((int)blockDim.x / tiles, Z));
+    const int per = (Z + parts - 1) / parts;
+    if ((int)threadIdx.x < tiles * parts) {
+        const int part = threadIdx.x / tiles, r = threadIdx.x - part * tiles;
+        const int sg = r / CG, cg = r - sg * CG;
+        float acc[SR][4];
+#pragma unroll
+        for (int s = 0; s < SR; ++s)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[s][c] = 0.f;
+        const int k0 = part * per, k1 = min(Z, k0 + per);
+        const float *__restrict__ W = a.head.W1 + 4 * cg;
+        const float *zrow = zt + sg * SR;
+#pragma unroll 4
+        for (int k = k0; k < k1; ++k) {
+            const float4 w = __ldg(reinterpret_cast<const float4 *>(W + (size_t)k * Hd));
+            float zv[SR];
+            if (SR == 4) {
+                const float4 t = *reinterpret_cast<const float4 *>(zrow + k * HS);
+                zv[0] = t.x; zv[1 % SR] = t.y; zv[2 % SR] = t.z; zv[3 % SR] = t.w;
+            } else if (SR == 2) {
+                const float2 t = *reinterpret_cast<const float2 *>(zrow + k * HS);
+                zv[0] = t.x; zv[1 % SR] = t.y;
+            } else {
+                zv[0] = zrow[k * HS];
+            }
+#pragma unroll
+            for (int s = 0; s < SR; ++s) {
+                acc[s][0] = fmaf(zv[s], w.x, acc[s][0]); acc[s][1] = fmaf(zv[s], w.y, acc[s][1]);
+                acc[s][2] = fmaf(zv[s], w.z, acc[s][2]); acc[s][3] = fmaf(zv[s], w.w, acc[s][3]);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int s = 0; s < SR; ++s)
+                red[((size_t)part * Hd + 4 * cg + c) * HS + sg * SR + s] = acc[s][c];
+    }
+    __syncthreads();
+    const bool relu = a.head.act == 0;
+    for (int i = threadIdx.x; i < Hd * HS; i += blockDim.x) {
+        float acc = a.head.b1[i / HS];
+        for (int q = 0; q < parts; ++q) acc += red[(size_t)q * Hd * HS + i];
+        hid[i] = relu ? fmaxf(acc, 0.f) : acc;
+    }
+    __syncthreads();
+    // head, second layer: one warp per (state, device)
+    {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+        for (int item = warp; item < HS * m; item += nw) {
+            const int s = item / m, j = item - s * m;
+            float acc = 0.f;
+            for (int k = lane; k < Hd; k += 32) acc = fmaf(hid[k * HS + s], a.head.W2[(size_t)k * m + j], acc);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            acc += a.head.b2[j];
+            if (lane == 0) lg[s * m + j] = (relu && a.head.final_act) ? fmaxf(acc, 0.f) : acc;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < HS && b0 + threadIdx.x < B) {
+        const int b = b0 + threadIdx.x;
+        const float *l = lg + threadIdx.x * m;
+        const int c = a.cur[b];
+        // a current node out of range yields NaN (ReLU would swallow a NaN input)
+        const bool valid = c >= 0 && c < a.n;
+        float mx = l[0];
+        for (int k = 1; k < m; ++k) mx = fmaxf(mx, l[k]);
+        float tot = 0.f;
+        for (int k = 0; k < m; ++k) tot += expf(l[k] - mx);
+        for (int k = 0; k < m; ++k) {
+            a.logits[(size_t)b * m + k] = valid ? l[k] : nanf("");
+            if (a.probs) a.probs[(size_t)b * m + k] = valid ? expf(l[k] - mx) / tot : nanf("");
+        }
+    }
+}
+
+bool head_fast_applicable(const PoolArgs &a) {
+    if ((a.d & 3) || a.head.n_layers != 2 || (a.head.hidden_dim & 3)) return false;
+    if (a.head.hidden_dim / 4 * 2 > kFastThreads) return false;
+    for (int i = 0; i < 3; ++i)
+        if (a.h[i].n_layers != 1 || a.h[i].in_dim != a.d || a.h[i].out_dim != a.d) return false;
+    return true;
+}
+
+template <int HS>
+cudaError_t launch_head_fast(const PoolArgs &a, cudaStream_t stream) {
+    const int Z = 5 * a.d + a.F, Hd = a.head.hidden_dim;
+    constexpr int SR = HS < 4 ? HS : 4;
+    const int tiles = (HS / SR) * (Hd / 4);
+    const int parts = std::max(1, std::min(kFastThreads / tiles, Z));
+    const size_t floats = (size_t)Z * HS + (size_t)HS * 3 * a.d + (size_t)Hd * HS + ((HS * a.m + 3) & ~3) +
+                          (size_t)parts * Hd * HS;
+    const size_t bytes = floats * sizeof(float);
+    if (bytes > 200 * 1024) return cudaErrorNotSupported;
+    cudaError_t err = cudaFuncSetAttribute(pool_head_fast_kernel<HS>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (err != cudaSuccess) return err;
+    // always preceded by one of this library's pooling kernels on the same stream
+    err = launch_overlapped(true, pool_head_fast_kernel<HS>, dim3((a.B + HS - 1) / HS), dim3(kFastThreads),
+                            bytes, stream, a);
+    count_launch();
+    return err;
+}
+
 }  // namespace
 
 int pool_chunks(int n, int B, const DeviceInfo &di) {
@@ -390,10 +577,18 @@ cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaS
     count_launch();
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    return launch_pool_head(a, stream);
+    return launch_pool_head(a, di, stream);
 }
 
-cudaError_t launch_pool_head(const PoolArgs &a, cudaStream_t stream) {
+cudaError_t launch_pool_head(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream) {
+    if (head_fast_applicable(a)) {
+        // fewest states per block that keeps the grid within two blocks per SM
+        const int limit = 2 * std::max(1, di.sm_count);
+        cudaError_t e = (a.B + 1) / 2 <= limit   ? launch_head_fast<2>(a, stream)
+                        : (a.B + 3) / 4 <= limit ? launch_head_fast<4>(a, stream)
+                                                 : launch_head_fast<8>(a, stream);
+        if (e != cudaErrorNotSupported) return e;
+    }
     const int Z = 5 * a.d + a.F;
     int tmp_floats = a.head.n_layers == 2 ? a.head.hidden_dim : 0;
     for (int i = 0; i < 3; ++i)
