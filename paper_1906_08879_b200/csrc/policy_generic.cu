@@ -384,17 +384,17 @@ pool_head_fast_kernel(const PoolArgs a) {
     for (int i = threadIdx.x; i < HS * 3 * d; i += blockDim.x) {
         const int s = i / (3 * d), j = i - s * 3 * d;
         const int b = min(b0 + s, B - 1);          // rows past the batch repeat the last state
-        // chunks are added in ascending order; four loads in flight at a time
+        // chunks are added in ascending order; eight loads in flight at a time
         const float *src = a.partial + (size_t)b * 3 * d + j;
         const size_t step = (size_t)B * 3 * d;
         float acc = 0.f;
-        int ch = 0;
-        for (; ch + 4 <= a.chunks; ch += 4) {
-            const float t0 = src[ch * step], t1 = src[(ch + 1) * step];
-            const float t2 = src[(ch + 2) * step], t3 = src[(ch + 3) * step];
-            acc = (((acc + t0) + t1) + t2) + t3;
+        for (int ch = 0; ch < a.chunks; ch += 8) {
+            float t[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) t[q] = ch + q < a.chunks ? src[(ch + q) * step] : 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc += t[q];
         }
-        for (; ch < a.chunks; ++ch) acc += src[ch * step];
         sum[i] = acc;
     }
     for (int i = threadIdx.x; i < HS * E; i += blockDim.x) {
@@ -418,12 +418,18 @@ pool_head_fast_kernel(const PoolArgs a) {
         const float *__restrict__ W = nt.W1 + 4 * cq;
         const float *v = sum + s * 3 * d + set * d;
         float4 acc = *reinterpret_cast<const float4 *>(nt.b1 + 4 * cq);
-#pragma unroll 8
-        for (int k = 0; k < d; ++k) {
-            const float4 w = __ldg(reinterpret_cast<const float4 *>(W + (size_t)k * d));
-            const float x = v[k];
-            acc.x = fmaf(x, w.x, acc.x); acc.y = fmaf(x, w.y, acc.y);
-            acc.z = fmaf(x, w.z, acc.z); acc.w = fmaf(x, w.w, acc.w);
+        for (int kb = 0; kb < d; kb += 16) {   // sixteen weight rows in flight (d is a multiple of 4)
+            float4 w[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t)
+                w[t] = kb + t < d ? __ldg(reinterpret_cast<const float4 *>(W + (size_t)(kb + t) * d))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const float x = kb + t < d ? v[kb + t] : 0.f;
+                acc.x = fmaf(x, w[t].x, acc.x); acc.y = fmaf(x, w[t].y, acc.y);
+                acc.z = fmaf(x, w[t].z, acc.z); acc.w = fmaf(x, w[t].w, acc.w);
+            }
         }
         if (nt.act == 0 && nt.final_act) {
             acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f);
@@ -448,23 +454,32 @@ pool_head_fast_kernel(const PoolArgs a) {
         const int k0 = part * per, k1 = min(Z, k0 + per);
         const float *__restrict__ W = a.head.W1 + 4 * cg;
         const float *zrow = zt + sg * SR;
-#pragma unroll 4
-        for (int k = k0; k < k1; ++k) {
-            const float4 w = __ldg(reinterpret_cast<const float4 *>(W + (size_t)k * Hd));
-            float zv[SR];
-            if (SR == 4) {
-                const float4 t = *reinterpret_cast<const float4 *>(zrow + k * HS);
-                zv[0] = t.x; zv[1 % SR] = t.y; zv[2 % SR] = t.z; zv[3 % SR] = t.w;
-            } else if (SR == 2) {
-                const float2 t = *reinterpret_cast<const float2 *>(zrow + k * HS);
-                zv[0] = t.x; zv[1 % SR] = t.y;
-            } else {
-                zv[0] = zrow[k * HS];
-            }
+        for (int kb = k0; kb < k1; kb += 16) {   // sixteen weight rows in flight
+            float4 w[16];
 #pragma unroll
-            for (int s = 0; s < SR; ++s) {
-                acc[s][0] = fmaf(zv[s], w.x, acc[s][0]); acc[s][1] = fmaf(zv[s], w.y, acc[s][1]);
-                acc[s][2] = fmaf(zv[s], w.z, acc[s][2]); acc[s][3] = fmaf(zv[s], w.w, acc[s][3]);
+            for (int t = 0; t < 16; ++t)
+                w[t] = kb + t < k1 ? __ldg(reinterpret_cast<const float4 *>(W + (size_t)(kb + t) * Hd))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const bool live = kb + t < k1;
+                const int k = live ? kb + t : k0;
+                float zv[SR];
+                if (SR == 4) {
+                    const float4 u = *reinterpret_cast<const float4 *>(zrow + k * HS);
+                    zv[0] = u.x; zv[1 % SR] = u.y; zv[2 % SR] = u.z; zv[3 % SR] = u.w;
+                } else if (SR == 2) {
+                    const float2 u = *reinterpret_cast<const float2 *>(zrow + k * HS);
+                    zv[0] = u.x; zv[1 % SR] = u.y;
+                } else {
+                    zv[0] = zrow[k * HS];
+                }
+#pragma unroll
+                for (int s = 0; s < SR; ++s) {
+                    zv[s] = live ? zv[s] : 0.f;
+                    acc[s][0] = fmaf(zv[s], w[t].x, acc[s][0]); acc[s][1] = fmaf(zv[s], w[t].y, acc[s][1]);
+                    acc[s][2] = fmaf(zv[s], w[t].z, acc[s][2]); acc[s][3] = fmaf(zv[s], w[t].w, acc[s][3]);
+                }
             }
         }
 #pragma unroll
