@@ -335,6 +335,61 @@ def test_two_streams_with_their_own_workspaces_do_not_interfere():
         assert torch.equal(logits, ref["logits"]) and torch.equal(probs, ref["probs"])
 
 
+def test_back_to_back_calls_with_inputs_changed_on_the_stream():
+    """The kernels of one forward call overlap their set-up with the kernel
+    before them. Nothing may be read early that an earlier kernel on the stream
+    still writes: states and weights are rewritten by ordinary stream work between
+    calls that share one workspace, and every call must see exactly its own."""
+    cfg = configs.make("inception")
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    B, m, n = cfg["B"], cfg["m"], cfg["n"]
+    r = rng(11)
+    variants = [states.random_states(r, n, m, B) for _ in range(3)]
+    cost, nbytes = dev_t(cfg["cost"]), dev_t(cfg["bytes"])
+    originals = [t.clone() for t in w._keep]
+
+    def set_weights(scale):
+        for t, o in zip(w._keep, originals):
+            t.copy_(o * scale)
+
+    # one call at a time, synchronised: the expected results
+    want = []
+    for k, (devs, cur, placed) in enumerate(variants):
+        set_weights(1.0 + 0.25 * k)
+        torch.cuda.synchronize()
+        lg, pr = placeto.placeto_policy_forward(g, w, cost, nbytes, dev_t(devs), dev_t(cur), dev_t(placed))
+        torch.cuda.synchronize()
+        want.append((lg.clone(), pr.clone()))
+    # the same calls queued back to back on one stream with one workspace and one set of buffers
+    ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD)
+    d_dev = torch.empty((B, n), dtype=torch.uint8, device="cuda")
+    d_cur = torch.empty((B,), dtype=torch.int32, device="cuda")
+    d_placed = torch.empty((B, n), dtype=torch.uint8, device="cuda")
+    staged = [(dev_t(a), dev_t(b), dev_t(c)) for a, b, c in variants]
+    got = []
+    torch.cuda.synchronize()
+    for k, (a, b, c) in enumerate(staged):
+        set_weights(1.0 + 0.25 * k)
+        d_dev.copy_(a); d_cur.copy_(b); d_placed.copy_(c)
+        lg = torch.empty((B, m), device="cuda")
+        pr = torch.empty((B, m), device="cuda")
+        placeto.placeto_policy_forward(g, w, cost, nbytes, d_dev, d_cur, d_placed, lg, pr, ws)
+        got.append((lg, pr))
+    torch.cuda.synchronize()
+    for (lg, pr), (wl, wp) in zip(got, want):
+        assert torch.equal(lg, wl) and torch.equal(pr, wp)
+
+
+@pytest.mark.parametrize("B", [593, 1185])
+def test_head_kernel_with_four_and_eight_states_per_block(B):
+    """Batches beyond two blocks per SM at two states per block move the head
+    kernel to four, then eight states per block."""
+    r = rng(B)
+    src, dst = random_dag(r, 20, 0.2)
+    _small_case(20, src, dst, d=32, m=4, B=B, seed=B)
+
+
 # ---------------------------------------------------------- error handling ---
 
 def test_argument_errors_are_reported_not_faulted():
