@@ -166,7 +166,8 @@ typedef enum {
     PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */
     PLACETO_CALL_LOGITS = 1,      /* placeto_policy_logits */
     PLACETO_CALL_FORWARD = 2,     /* placeto_policy_forward */
-    PLACETO_CALL_FORWARD_HOST = 3 /* placeto_policy_forward_host */
+    PLACETO_CALL_FORWARD_HOST = 3,/* placeto_policy_forward_host */
+    PLACETO_CALL_EPISODE = 4      /* placeto_episode_rollout (B = number of episodes) */
 } placeto_call;
 
 /* Bytes of DEVICE workspace `call` needs for batch size B (0 on invalid arguments).
@@ -236,6 +237,38 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
                                            const uint8_t *placed, int32_t B, float *logits,
                                            float *probs, void *workspace, size_t workspace_bytes,
                                            uint32_t flags, void *stream);
+
+/*
+ * A whole placement episode per call, for E independent episodes on one graph
+ * (the MDP of Sec. 2.1 of the paper driven by the policy of Sec. 2.2): for
+ * t = 0 .. n-1 the node order[t] is current; the policy is evaluated on the E
+ * current states (features, both passes, pooling, head: the same kernels as
+ * placeto_policy_forward); every episode picks a device for its current node;
+ * the node takes that device and is marked visited. Visited flags start at 0 and
+ * the current node itself counts as not yet visited. All steps are queued on
+ * `stream` without a host round trip: n * (policy kernels + one transition kernel).
+ *
+ * cost, bytes : DEVICE float[n].
+ * order       : DEVICE int32[n], the visiting order, a permutation of 0 .. n-1 (the
+ *               paper leaves the order arbitrary). Not checked: an id outside
+ *               [0, n) makes that step's policy output NaN and leaves the
+ *               placement untouched; a repeated id is visited twice.
+ * uniforms    : NULL for greedy episodes (largest logit, lowest device among equals),
+ *               else DEVICE float[E][n] of numbers in [0, 1): step t of episode e takes
+ *               the first device k with p_0 + .. + p_k > uniforms[e][t], p = softmax(logits).
+ * dev         : DEVICE uint8[E][n], in: the initial placement (devices < m); out: the
+ *               final one (every node carries the device chosen at its step).
+ * actions     : DEVICE uint8[E][n] or NULL, the device chosen at step t (by step, not by node).
+ * logp        : DEVICE float[E][n] or NULL, log pi(action | state) of step t.
+ * workspace   : DEVICE, at least placeto_workspace_bytes(g, w, E, PLACETO_CALL_EPISODE, flags).
+ * Requires w->F == w->m + 4. Errors as for placeto_policy_forward.
+ */
+placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_weights *w,
+                                       const float *cost, const float *bytes,
+                                       const int32_t *order, const float *uniforms, int32_t E,
+                                       uint8_t *dev, uint8_t *actions, float *logp,
+                                       void *workspace, size_t workspace_bytes, uint32_t flags,
+                                       void *stream);
 
 /*
  * placeto_policy_logits without a workspace argument, for callers that must not

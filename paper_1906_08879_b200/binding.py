@@ -21,14 +21,14 @@ LIB_PATH = os.path.join(_HERE, "libplaceto.so")
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
 PLACETO_FMA_ONLY, PLACETO_TENSOR = 16, 32
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
-CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST = 0, 1, 2, 3
+CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "placeto_status_string", "placeto_graph_create", "placeto_graph_info",
     "placeto_graph_host_view", "placeto_graph_destroy", "placeto_workspace_bytes",
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
-    "placeto_last_launch_count",
+    "placeto_episode_rollout", "placeto_last_launch_count",
 )
 
 
@@ -75,7 +75,7 @@ def _load() -> ctypes.CDLL:
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
-                 "placeto_policy_logits_static"):
+                 "placeto_policy_logits_static", "placeto_episode_rollout"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -310,6 +310,26 @@ def placeto_policy_logits_static(g: Graph, w: Weights, X, H_down, H_up, cur, log
                                              _p(probs), ctypes.c_uint32(flags), _stream(stream)),
            "placeto_policy_logits_static")
     return logits, probs
+
+
+def placeto_episode_rollout(g: Graph, w: Weights, cost, nbytes, order, dev, uniforms=None,
+                            actions=None, logp=None, ws=None, flags: int = 0, stream=None):
+    """E = dev.shape[0] episodes over the graph; `dev` (uint8 [E][n]) holds the
+    initial placement and is overwritten with the final one. `uniforms` (float
+    [E][n]) switches from greedy to sampled choices. Returns (dev, actions, logp)."""
+    E = dev.shape[0]
+    if actions is None:
+        actions = torch.empty((E, g.n), dtype=torch.uint8, device=dev.device)
+    if logp is None:
+        logp = torch.empty((E, g.n), dtype=torch.float32, device=dev.device)
+    if ws is None:
+        ws = workspace(g, w, E, CALL_EPISODE, flags, dev.device)
+    _check(_lib.placeto_episode_rollout(g.handle, ctypes.byref(w.c), _p(cost), _p(nbytes), _p(order),
+                                        _p(uniforms), ctypes.c_int32(E), _p(dev), _p(actions),
+                                        _p(logp), _p(ws), ctypes.c_size_t(ws.numel()),
+                                        ctypes.c_uint32(flags), _stream(stream)),
+           "placeto_episode_rollout")
+    return dev, actions, logp
 
 
 def placeto_last_launch_count() -> int:

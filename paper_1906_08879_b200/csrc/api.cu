@@ -112,6 +112,12 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         L.logits = take((size_t)B * m * sizeof(float));
         L.probs = take((size_t)B * m * sizeof(float));
     }
+    if (call == PLACETO_CALL_EPISODE) {
+        L.placed = take(n * B);
+        L.cur = take((size_t)B * sizeof(int32_t));
+        L.logits = take((size_t)B * m * sizeof(float));
+        L.probs = take((size_t)B * m * sizeof(float));
+    }
     L.total = off;
     return L;
 }
@@ -360,7 +366,7 @@ void placeto_graph_destroy(placeto_graph *g) {
 size_t placeto_workspace_bytes(const placeto_graph *g, const placeto_weights *w, int32_t B,
                                placeto_call call, uint32_t flags) {
     if (!g || !w || B < 1 || !flags_ok(flags) || dims_ok(w) != PLACETO_OK) return 0;
-    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_FORWARD_HOST) return 0;
+    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_EPISODE) return 0;
     placeto_graph tmp_info;   // HOST_ONLY graphs have no device info: assume a full B200
     const placeto_graph *use = g;
     if (!g->on_device) {
@@ -525,6 +531,52 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
     if (!scratch) return PLACETO_ERR_CUDA;
     return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, scratch, L, flags,
                     static_cast<cudaStream_t>(stream));
+}
+
+placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_weights *w,
+                                       const float *cost, const float *bytes,
+                                       const int32_t *order, const float *uniforms, int32_t E,
+                                       uint8_t *dev, uint8_t *actions, float *logp,
+                                       void *workspace, size_t workspace_bytes, uint32_t flags,
+                                       void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s == PLACETO_OK) s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (E < 1 || w->m > PLACETO_MAX_M || w->F != w->m + 4) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, E, PLACETO_CALL_EPISODE);
+    s = common_checks(g, E, workspace, workspace_bytes, L.total, flags);
+    if (s != PLACETO_OK) return s;
+    if (!cost || !bytes || !order || !dev) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(order) || !aligned16(dev) ||
+        (uniforms && !aligned16(uniforms)) || (actions && !aligned16(actions)) ||
+        (logp && !aligned16(logp)))
+        return PLACETO_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float *X = reinterpret_cast<float *>(ws + L.X);
+    float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
+    float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
+    EpisodeArgs ep;
+    ep.n = g->host.n; ep.E = E; ep.m = w->m;
+    ep.order = order; ep.uniforms = uniforms;
+    ep.logits = reinterpret_cast<float *>(ws + L.logits);
+    ep.dev = dev;
+    ep.placed = reinterpret_cast<uint8_t *>(ws + L.placed);
+    ep.cur = reinterpret_cast<int32_t *>(ws + L.cur);
+    ep.logp = logp; ep.actions = actions;
+    float *probs = reinterpret_cast<float *>(ws + L.probs);
+    s = cuda_status(launch_episode_begin(ep, st));
+    for (int t = 0; s == PLACETO_OK && t < ep.n; ++t) {
+        // one policy evaluation of the E current states, then the transition
+        s = cuda_status(launch_features(ep.n, E, w->m, cost, bytes, dev, ep.cur, ep.placed, X, st));
+        if (s == PLACETO_OK) s = run_embed(g, w, X, E, Hd, Hu, ws, L, flags, st, true);
+        if (s == PLACETO_OK)
+            s = run_pool(g, w, X, Hd, Hu, ep.cur, E, const_cast<float *>(ep.logits), probs, ws, L, flags, st, true);
+        if (s == PLACETO_OK) s = cuda_status(launch_episode_step(ep, t, st));
+    }
+    return s;
 }
 
 int32_t placeto_last_launch_count(void) { return t_launches; }

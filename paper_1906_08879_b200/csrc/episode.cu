@@ -1,0 +1,83 @@
+// The MDP transition of a placement episode (Sec. 2.1 of the Placeto paper) on
+// the device: after the policy kernels have produced the logits of step t, one
+// thread per episode picks the current node's device (argmax, or an inverse-CDF
+// sample driven by a caller-supplied uniform number), writes it into the
+// placement, marks the node visited, records the log-probability of the choice
+// and makes the next node of the visiting order current. With it a whole episode
+// runs as a stream of launches without a host round trip per step.
+#include <cmath>
+
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kThreads = 128;
+
+// placed[e][:] = 0 and cur[e] = order[0] for every episode
+__global__ void episode_begin_kernel(int n, int E, const int *__restrict__ order,
+                                     uint8_t *__restrict__ placed, int *__restrict__ cur) {
+    const size_t total = (size_t)E * n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x)
+        placed[i] = 0;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < E) cur[e] = order[0];
+}
+
+// Greedy: the largest logit, the lowest index among equals. Sampling: with
+// p = softmax(logits) (max-subtracted, FP32, summed in index order), the first
+// index k with p_0 + .. + p_k > u, the last index if rounding leaves none.
+__global__ void episode_step_kernel(EpisodeArgs a, int t) {
+    dependents_may_start();
+    dependency_wait();          // the logits come from a kernel that may still be running
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= a.E) return;
+    const int m = a.m, n = a.n;
+    const float *l = a.logits + (size_t)e * m;
+    const int v = a.order[t];
+    float mx = l[0];
+    int best = 0;
+    for (int k = 1; k < m; ++k)
+        if (l[k] > mx) { mx = l[k]; best = k; }
+    float tot = 0.f;
+    for (int k = 0; k < m; ++k) tot += expf(l[k] - mx);
+    int action = best;
+    if (a.uniforms != nullptr) {
+        const float u = a.uniforms[(size_t)e * n + t];
+        float cum = 0.f;
+        action = m - 1;
+        for (int k = 0; k < m; ++k) {
+            cum += expf(l[k] - mx) / tot;
+            if (cum > u) { action = k; break; }
+        }
+    }
+    if (a.logp != nullptr) a.logp[(size_t)e * n + t] = (l[action] - mx) - logf(tot);
+    if (a.actions != nullptr) a.actions[(size_t)e * n + t] = (uint8_t)action;
+    if (v >= 0 && v < n) {      // an id outside the graph leaves the placement alone
+        a.dev[(size_t)e * n + v] = (uint8_t)action;
+        a.placed[(size_t)e * n + v] = 1;
+    }
+    if (t + 1 < n) a.cur[e] = a.order[t + 1];
+}
+
+}  // namespace
+
+cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream) {
+    const int blocks = std::max(1, std::min(1024, (int)(((size_t)a.E * a.n + kThreads - 1) / kThreads)));
+    const int need = (a.E + kThreads - 1) / kThreads;       // every episode needs its thread
+    episode_begin_kernel<<<std::max(blocks, need), kThreads, 0, stream>>>(a.n, a.E, a.order, a.placed, a.cur);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream) {
+    // always preceded by this library's head kernel on the same stream
+    cudaError_t err = launch_overlapped(true, episode_step_kernel, dim3((a.E + kThreads - 1) / kThreads),
+                                        dim3(kThreads), 0, stream, a, t);
+    count_launch();
+    return err;
+}
+
+}  // namespace placeto

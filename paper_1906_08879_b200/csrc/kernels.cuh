@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstddef>
 #include <cstdint>
 
@@ -65,6 +66,17 @@ struct PoolArgs {
     int chunks, chunk_nodes;
 };
 
+struct EpisodeArgs {
+    int n, E, m;
+    const int *order;          // [n] node visited at step t
+    const float *uniforms;     // [E][n] or null (greedy)
+    const float *logits;       // [E][m] of the current step
+    uint8_t *dev, *placed;     // [E][n]
+    int *cur;                  // [E]
+    float *logp;               // [E][n] by step, or null
+    uint8_t *actions;          // [E][n] by step, or null
+};
+
 struct DeviceInfo {
     int sm_count;
     int max_smem_optin;   // bytes per block
@@ -107,6 +119,10 @@ cudaError_t launch_overlapped(bool overlap, void (*kern)(KArgs...), dim3 grid, d
 cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
                             cudaStream_t stream);
+
+// episode.cu: the MDP transition between two policy evaluations of an episode
+cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream);
+cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream);
 
 // embed_generic.cu: dimension-generic message passing. schedule is one of
 // PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.
