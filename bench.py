@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--flags", type=int, default=0, help="schedule flags of placeto.h")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0)
+    ap.add_argument("--episodes", type=int, default=0,
+                    help="E > 0: a step is one placeto_episode_rollout call of E sampled episodes over the "
+                         "workload's graph (|V| policy evaluations per episode, transitions on the device)")
     return ap.parse_args()
 
 
@@ -246,7 +249,13 @@ def run_b200(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     cfg = make_workload(args.workload, rank)
+    if args.episodes > 0:   # E states per policy evaluation: the current states of the E episodes
+        from gen import states as gen_states
+        rng_e = np.random.Generator(np.random.PCG64(4242 + rank))
+        cfg["dev"], cfg["cur"], cfg["placed"] = gen_states.random_states(rng_e, cfg["n"], cfg["m"], args.episodes)
+        cfg["B"] = args.episodes
     n, B, m, d, F = cfg["n"], cfg["B"], cfg["m"], cfg["d"], cfg["F"]
+    units = B * n if args.episodes > 0 else B      # policy evaluations per step
     g = placeto.Graph(n, cfg["src"], cfg["dst"])
     w = placeto.Weights(cfg["weights"])
     dev_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
@@ -258,7 +267,21 @@ def run_b200(args):
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
 
+    if args.episodes > 0:
+        from gen import graphs as gen_graphs
+        order = dev_t(gen_graphs.topological_order(n, cfg["src"], cfg["dst"]))
+        uniforms = dev_t(rng_e.random(size=(B, n)).astype(np.float32))
+        dev0 = devs.clone()
+        actions = torch.empty((B, n), dtype=torch.uint8, device="cuda")
+        logp = torch.empty((B, n), dtype=torch.float32, device="cuda")
+        ws_ep = placeto.workspace(g, w, B, placeto.CALL_EPISODE, args.flags)
+
     def step():
+        if args.episodes > 0:
+            devs.copy_(dev0)
+            placeto.placeto_episode_rollout(g, w, cost, nbytes, order, devs, uniforms, actions, logp,
+                                            ws_ep, args.flags, stream)
+            return
         placeto.placeto_policy_forward(g, w, cost, nbytes, devs, cur, placed, logits, probs, ws,
                                        args.flags, stream)
 
@@ -293,7 +316,7 @@ def run_b200(args):
     total_ms, launches = timed(step, args.steps, count_launches=True)
     barrier()
     clocks = sampler.stop()
-    value, total_ms = job_throughput(total_ms, B, args.steps, dist, "cuda")
+    value, total_ms = job_throughput(total_ms, units, args.steps, dist, "cuda")
 
     # end to end through the host-buffer entry point: pinned inputs -> device -> results on host
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -301,7 +324,20 @@ def run_b200(args):
     h_logits = torch.empty((B, m), dtype=torch.float32).pin_memory()
     h_probs = torch.empty((B, m), dtype=torch.float32).pin_memory()
 
+    if args.episodes > 0:
+        h_dev0 = pin(cfg["dev"])
+        h_actions = torch.empty((B, n), dtype=torch.uint8).pin_memory()
+        h_logp = torch.empty((B, n), dtype=torch.float32).pin_memory()
+
     def e2e_step():
+        if args.episodes > 0:   # initial placement in, actions and log-probabilities out
+            devs.copy_(h_dev0, non_blocking=True)
+            placeto.placeto_episode_rollout(g, w, cost, nbytes, order, devs, uniforms, actions, logp,
+                                            ws_ep, args.flags, stream)
+            h_actions.copy_(actions, non_blocking=True)
+            h_logp.copy_(logp, non_blocking=True)
+            stream.synchronize()
+            return
         placeto.placeto_policy_forward_host(g, w, *h_in, h_logits, h_probs, ws, args.flags, stream)
 
     for _ in range(3):
@@ -309,10 +345,14 @@ def run_b200(args):
     barrier()
     e2e_ms, _ = timed(e2e_step, args.steps)
     barrier()
-    e2e_value, _ = job_throughput(e2e_ms, B, args.steps, dist, "cuda")
+    e2e_value, _ = job_throughput(e2e_ms, units, args.steps, dist, "cuda")
     h2d = sum(x.numel() * x.element_size() for x in h_in)
     d2h = h_logits.numel() * 4 + h_probs.numel() * 4
-    assert torch.equal(h_logits.cuda(), logits), "host and device entry points disagree"
+    if args.episodes > 0:
+        h2d, d2h = h_dev0.numel(), h_actions.numel() + 4 * h_logp.numel()
+        assert torch.equal(h_actions.cuda(), actions), "host copy of the actions differs"
+    else:
+        assert torch.equal(h_logits.cuda(), logits), "host and device entry points disagree"
 
     # the dominant kernel alone: the message-passing launch(es) of embed_forward
     X = placeto.placeto_build_features(g, cost, nbytes, devs, cur, placed, m)
@@ -368,10 +408,15 @@ def run_b200(args):
 
     cores = len(os.sched_getaffinity(0))
     cpu_value, cpu_s, passes = time_oracle(cfg, args.cpu_baseline_seconds, cores)
+    config = workload_config(cfg, world)
+    if args.episodes > 0:
+        config.update(workload=cfg["name"] + "-episodes", episodes_per_gpu=B, steps_per_episode=n,
+                      choice="sampled (inverse CDF of the device softmax)",
+                      l2="flushed between timed rollouts only (256 MiB memset, outside the timed events)")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, world), "clocks": clocks,
+            "config": config, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches, "roofline": roofline,
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
