@@ -247,6 +247,7 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
  * the node takes that device and is marked visited. Visited flags start at 0 and
  * the current node itself counts as not yet visited. All steps are queued on
  * `stream` without a host round trip: n * (policy kernels + one transition kernel).
+ * The feature tensor is built once; a transition patches the two rows it changes.
  *
  * cost, bytes : DEVICE float[n].
  * order       : DEVICE int32[n], the visiting order, a permutation of 0 .. n-1 (the

@@ -567,11 +567,14 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
     ep.cur = reinterpret_cast<int32_t *>(ws + L.cur);
     ep.logp = logp; ep.actions = actions;
     float *probs = reinterpret_cast<float *>(ws + L.probs);
+    ep.X = X;
     s = cuda_status(launch_episode_begin(ep, st));
+    // the features of the initial states; every later step patches them in place
+    if (s == PLACETO_OK)
+        s = cuda_status(launch_features(ep.n, E, w->m, cost, bytes, dev, ep.cur, ep.placed, X, st));
     for (int t = 0; s == PLACETO_OK && t < ep.n; ++t) {
         // one policy evaluation of the E current states, then the transition
-        s = cuda_status(launch_features(ep.n, E, w->m, cost, bytes, dev, ep.cur, ep.placed, X, st));
-        if (s == PLACETO_OK) s = run_embed(g, w, X, E, Hd, Hu, ws, L, flags, st, true);
+        s = run_embed(g, w, X, E, Hd, Hu, ws, L, flags, st, true);
         if (s == PLACETO_OK)
             s = run_pool(g, w, X, Hd, Hu, ep.cur, E, const_cast<float *>(ep.logits), probs, ws, L, flags, st, true);
         if (s == PLACETO_OK) s = cuda_status(launch_episode_step(ep, t, st));

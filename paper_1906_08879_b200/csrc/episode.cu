@@ -4,7 +4,11 @@
 // sample driven by a caller-supplied uniform number), writes it into the
 // placement, marks the node visited, records the log-probability of the choice
 // and makes the next node of the visiting order current. With it a whole episode
-// runs as a stream of launches without a host round trip per step.
+// runs as a stream of launches without a host round trip per step. A step changes
+// the raw features of two nodes only (the node just placed: device one-hot,
+// current flag off, visited flag on; the next node: current flag on), so the
+// same thread patches those rows of X in place and the feature tensor is built
+// once per episode, not once per step.
 #include <cmath>
 
 #include "kernels.cuh"
@@ -55,11 +59,20 @@ __global__ void episode_step_kernel(EpisodeArgs a, int t) {
     }
     if (a.logp != nullptr) a.logp[(size_t)e * n + t] = (l[action] - mx) - logf(tot);
     if (a.actions != nullptr) a.actions[(size_t)e * n + t] = (uint8_t)action;
+    const int F = m + 4;        // x = [cost, bytes, one-hot(m), is-current, is-visited]
     if (v >= 0 && v < n) {      // an id outside the graph leaves the placement alone
         a.dev[(size_t)e * n + v] = (uint8_t)action;
         a.placed[(size_t)e * n + v] = 1;
+        float *x = a.X + ((size_t)v * a.E + e) * F;
+        for (int k = 0; k < m; ++k) x[2 + k] = k == action ? 1.f : 0.f;
+        x[2 + m] = 0.f;
+        x[3 + m] = 1.f;
     }
-    if (t + 1 < n) a.cur[e] = a.order[t + 1];
+    if (t + 1 < n) {
+        const int next = a.order[t + 1];
+        a.cur[e] = next;
+        if (next >= 0 && next < n) a.X[((size_t)next * a.E + e) * F + 2 + m] = 1.f;
+    }
 }
 
 }  // namespace

@@ -75,6 +75,7 @@ struct EpisodeArgs {
     int *cur;                  // [E]
     float *logp;               // [E][n] by step, or null
     uint8_t *actions;          // [E][n] by step, or null
+    float *X;                  // [n][E][m + 4] raw features, patched in place after every step
 };
 
 struct DeviceInfo {
