@@ -167,7 +167,8 @@ typedef enum {
     PLACETO_CALL_LOGITS = 1,      /* placeto_policy_logits */
     PLACETO_CALL_FORWARD = 2,     /* placeto_policy_forward */
     PLACETO_CALL_FORWARD_HOST = 3,/* placeto_policy_forward_host */
-    PLACETO_CALL_EPISODE = 4      /* placeto_episode_rollout (B = number of episodes) */
+    PLACETO_CALL_EPISODE = 4,     /* placeto_episode_rollout (B = number of episodes) */
+    PLACETO_CALL_EMBED_ROUNDS = 5 /* placeto_embed_rounds */
 } placeto_call;
 
 /* Bytes of DEVICE workspace `call` needs for batch size B (0 on invalid arguments).
@@ -237,6 +238,23 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
                                            const uint8_t *placed, int32_t B, float *logits,
                                            float *probs, void *workspace, size_t workspace_bytes,
                                            uint32_t flags, void *stream);
+
+/*
+ * Step 2 in the synchronous form the paper states (Sec. 2.2 step 2: the message
+ * passing updates are repeated k times, k a hyper-parameter): H^0 = 0 and, for
+ * r = 1 .. rounds, every node at once from the previous round's values,
+ *   H^r_v = g( sum_{u in nbr(v)} f([H^(r-1)_u || x_u]) ),
+ * top-down over parents into H_down and bottom-up over children into H_up, each
+ * with its own f and g. Output: H^rounds. For rounds >= depth of the graph the
+ * result equals placeto_embed_forward's (the progressive sweep is its fixed
+ * point); fewer rounds give the truncated, local summaries. rounds + 1 launches
+ * of the dimension-generic kernel; every width, depth and activation is accepted.
+ * X, H_down, H_up, B as for placeto_embed_forward; rounds >= 0 (0 gives zeros).
+ * workspace: DEVICE, at least placeto_workspace_bytes(.., PLACETO_CALL_EMBED_ROUNDS, 0).
+ */
+placeto_status placeto_embed_rounds(const placeto_graph *g, const placeto_weights *w, const float *X,
+                                    int32_t B, int32_t rounds, float *H_down, float *H_up,
+                                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * A whole placement episode per call, for E independent episodes on one graph

@@ -21,14 +21,14 @@ LIB_PATH = os.path.join(_HERE, "libplaceto.so")
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
 PLACETO_FMA_ONLY, PLACETO_TENSOR = 16, 32
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
-CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE = 0, 1, 2, 3, 4
+CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE, CALL_EMBED_ROUNDS = 0, 1, 2, 3, 4, 5
 
 EXPORTS = (
     "placeto_status_string", "placeto_graph_create", "placeto_graph_info",
     "placeto_graph_host_view", "placeto_graph_destroy", "placeto_workspace_bytes",
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
-    "placeto_episode_rollout", "placeto_last_launch_count",
+    "placeto_episode_rollout", "placeto_embed_rounds", "placeto_last_launch_count",
 )
 
 
@@ -75,7 +75,7 @@ def _load() -> ctypes.CDLL:
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
-                 "placeto_policy_logits_static", "placeto_episode_rollout"):
+                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -244,6 +244,23 @@ def placeto_embed_forward(g: Graph, w: Weights, X, H_down=None, H_up=None, ws=No
                                       _p(H_down), _p(H_up), _p(ws), ctypes.c_size_t(ws.numel()),
                                       ctypes.c_uint32(flags), _stream(stream)),
            "placeto_embed_forward")
+    return H_down, H_up
+
+
+def placeto_embed_rounds(g: Graph, w: Weights, X, rounds: int, H_down=None, H_up=None, ws=None,
+                         stream=None):
+    """The synchronous k-round form of the message passing (from zeros)."""
+    B = X.shape[1]
+    if H_down is None:
+        H_down = torch.empty((g.n, B, w.d), dtype=torch.float32, device=X.device)
+    if H_up is None:
+        H_up = torch.empty((g.n, B, w.d), dtype=torch.float32, device=X.device)
+    if ws is None:
+        ws = workspace(g, w, B, CALL_EMBED_ROUNDS, 0, X.device)
+    _check(_lib.placeto_embed_rounds(g.handle, ctypes.byref(w.c), _p(X), ctypes.c_int32(B),
+                                     ctypes.c_int32(rounds), _p(H_down), _p(H_up), _p(ws),
+                                     ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "placeto_embed_rounds")
     return H_down, H_up
 
 

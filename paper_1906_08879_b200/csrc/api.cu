@@ -74,7 +74,7 @@ placeto_status pool_weights_ok(const placeto_weights *w) {
 }
 
 struct Layout {
-    size_t msg[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
+    size_t msg[2], msg_alt[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
     int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
 };
@@ -88,17 +88,24 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
     int chunks = pool_chunks((int)n, B, g->info);
     L.chunk_nodes = ((int)n + chunks - 1) / chunks;
     L.chunks = ((int)n + L.chunk_nodes - 1) / L.chunk_nodes;
-    if (call == PLACETO_CALL_EMBED || call >= PLACETO_CALL_FORWARD) {
+    if (call == PLACETO_CALL_EMBED || call == PLACETO_CALL_EMBED_ROUNDS ||
+        (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE)) {
         L.msg[0] = take(n * B * d * sizeof(float));
         L.msg[1] = take(n * B * d * sizeof(float));
+    }
+    if (call == PLACETO_CALL_EMBED_ROUNDS) {
+        L.msg_alt[0] = take(n * B * d * sizeof(float));
+        L.msg_alt[1] = take(n * B * d * sizeof(float));
+        L.total = off;
+        return L;
     }
     if (w->F >= 4 && w->F <= 16 && (w->F & 3) == 0) {
         if (w->d == 32) pool_d32_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
         if (w->d == 64) pool_d64_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
     }
-    if (call == PLACETO_CALL_LOGITS || call >= PLACETO_CALL_FORWARD)
+    if (call == PLACETO_CALL_LOGITS || (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE))
         L.partial = take((size_t)std::max(L.chunks, L.chunks32) * B * 3 * d * sizeof(float));
-    if (call >= PLACETO_CALL_FORWARD) {
+    if (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE) {
         L.X = take(n * B * F * sizeof(float));
         L.H[0] = take(n * B * d * sizeof(float));
         L.H[1] = take(n * B * d * sizeof(float));
@@ -366,7 +373,7 @@ void placeto_graph_destroy(placeto_graph *g) {
 size_t placeto_workspace_bytes(const placeto_graph *g, const placeto_weights *w, int32_t B,
                                placeto_call call, uint32_t flags) {
     if (!g || !w || B < 1 || !flags_ok(flags) || dims_ok(w) != PLACETO_OK) return 0;
-    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_EPISODE) return 0;
+    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_EMBED_ROUNDS) return 0;
     placeto_graph tmp_info;   // HOST_ONLY graphs have no device info: assume a full B200
     const placeto_graph *use = g;
     if (!g->on_device) {
@@ -531,6 +538,42 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
     if (!scratch) return PLACETO_ERR_CUDA;
     return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, scratch, L, flags,
                     static_cast<cudaStream_t>(stream));
+}
+
+placeto_status placeto_embed_rounds(const placeto_graph *g, const placeto_weights *w, const float *X,
+                                    int32_t B, int32_t rounds, float *H_down, float *H_up,
+                                    void *workspace, size_t workspace_bytes, void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1 || rounds < 0) return PLACETO_ERR_INVALID_ARG;
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_EMBED_ROUNDS);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, 0);
+    if (s != PLACETO_OK) return s;
+    if (!X || !H_down || !H_up || !aligned16(X) || !aligned16(H_down) || !aligned16(H_up))
+        return PLACETO_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    EmbedArgs a;
+    a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
+    a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
+    a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
+    a.X = X;
+    a.H[0] = H_down; a.H[1] = H_up;
+    a.M[0] = a.M[1] = nullptr;
+    a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
+    a.max_level_width = g->host.max_level_width;
+    if (rounds == 0) {      // H^0 = 0
+        const size_t bytes = (size_t)a.n * B * a.d * sizeof(float);
+        if (cudaMemsetAsync(H_down, 0, bytes, st) != cudaSuccess ||
+            cudaMemsetAsync(H_up, 0, bytes, st) != cudaSuccess)
+            return PLACETO_ERR_CUDA;
+        return PLACETO_OK;
+    }
+    float *msg[4] = {reinterpret_cast<float *>(ws + L.msg[0]), reinterpret_cast<float *>(ws + L.msg_alt[0]),
+                     reinterpret_cast<float *>(ws + L.msg[1]), reinterpret_cast<float *>(ws + L.msg_alt[1])};
+    return cuda_status(launch_embed_rounds(a, g->info, rounds, msg, st));
 }
 
 placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_weights *w,

@@ -36,6 +36,12 @@ struct GenericPlan {
     int width;        // floats per buffered row
     int weights_in_smem;
     int level_begin, level_end;
+    // Synchronous rounds (all nodes at once from the previous round's messages):
+    // 0 off; 1 a round: h = g(sum of M_in), M_out = f([h || x]); 2 the start:
+    // h = 0 (not stored), M_out = f([0 || x]).
+    int round_mode;
+    const float *M_in[2];
+    float *M_out[2];
     size_t smem_bytes;
 };
 
@@ -80,7 +86,8 @@ embed_generic_kernel(const EmbedArgs a, const GenericPlan p) {
     const int d = a.d, F = a.F, B = a.B;
     const float *__restrict__ X = a.X;
     float *__restrict__ H = a.H[dir];
-    float *M = a.M[dir];
+    const float *Min = p.round_mode ? p.M_in[dir] : a.M[dir];
+    float *M = p.round_mode ? p.M_out[dir] : a.M[dir];
 
     // Stage the direction's weights once per block.
     const float *fW1 = f.W1, *fb1 = f.b1, *fW2 = f.W2, *fb2 = f.b2;
@@ -110,7 +117,9 @@ embed_generic_kernel(const EmbedArgs a, const GenericPlan p) {
     const int last = kCooperative ? p.level_end : min(p.level_end, lv.n_levels);
     for (int level = p.level_begin; level < last; ++level) {
         if (level < lv.n_levels) {
-            const int p0 = lv.level_ptr[level], p1 = lv.level_ptr[level + 1];
+            // a synchronous round treats all nodes as one level
+            const int p0 = p.round_mode ? 0 : lv.level_ptr[level];
+            const int p1 = p.round_mode ? a.n : lv.level_ptr[level + 1];
             const int width_l = p1 - p0;
             const int mine = (width_l - split + p.node_splits - 1) / p.node_splits;  // nodes p0+split+q*splits
             const int rows_total = mine > 0 ? mine * nb : 0;
@@ -122,19 +131,21 @@ embed_generic_kernel(const EmbedArgs a, const GenericPlan p) {
                     const int q = (r0 + r) / nb, b = b0 + (r0 + r) - q * nb;
                     const int pos = p0 + split + q * p.node_splits;
                     float s = 0.f;
-                    for (int e = lv.nbr_ptr[pos]; e < lv.nbr_ptr[pos + 1]; ++e)
-                        s += __ldcg(M + ((size_t)lv.nbr[e] * B + b) * d + j);
+                    if (p.round_mode != 2)
+                        for (int e = lv.nbr_ptr[pos]; e < lv.nbr_ptr[pos + 1]; ++e)
+                            s += __ldcg(Min + ((size_t)lv.nbr[e] * B + b) * d + j);
                     bufA[r * stride + j] = s;
                 }
                 __syncthreads();
-                float *h = apply_mlp(g, gW1, gb1, gW2, gb2, bufA, bufB, stride, rows);
+                float *h = p.round_mode == 2 ? bufA
+                                             : apply_mlp(g, gW1, gb1, gW2, gb2, bufA, bufB, stride, rows);
                 float *other = (h == bufA) ? bufB : bufA;
                 // store h and append the node's raw features: [h || x]
                 for (int idx = threadIdx.x; idx < rows * (d + F); idx += blockDim.x) {
                     const int r = idx / (d + F), j = idx - r * (d + F);
                     const int q = (r0 + r) / nb, b = b0 + (r0 + r) - q * nb;
                     const int v = lv.order[p0 + split + q * p.node_splits];
-                    if (j < d) H[((size_t)v * B + b) * d + j] = h[r * stride + j];
+                    if (j < d) { if (p.round_mode != 2) H[((size_t)v * B + b) * d + j] = h[r * stride + j]; }
                     else h[r * stride + j] = X[((size_t)v * B + b) * F + (j - d)];
                 }
                 __syncthreads();
@@ -156,8 +167,10 @@ int slices_for(int B, int target) { return std::max(1, std::min(B, target)); }
 
 }  // namespace
 
-cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,
-                                 cudaStream_t stream) {
+namespace {
+
+// Row buffers, weight staging and state slices common to every schedule.
+GenericPlan base_plan(const EmbedArgs &a, const DeviceInfo &di) {
     GenericPlan p;
     const int max_hidden = std::max(std::max(a.f[0].hidden_dim, a.f[1].hidden_dim),
                                     std::max(a.g[0].hidden_dim, a.g[1].hidden_dim));
@@ -183,6 +196,17 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
     p.S = (a.B + n_slices - 1) / n_slices;
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.node_splits = 1;
+    p.round_mode = 0;
+    p.M_in[0] = p.M_in[1] = nullptr;
+    p.M_out[0] = p.M_out[1] = nullptr;
+    return p;
+}
+
+}  // namespace
+
+cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,
+                                 cudaStream_t stream) {
+    GenericPlan p = base_plan(a, di);
     const int max_levels = std::max(a.lv[0].n_levels, a.lv[1].n_levels);
 
     cudaError_t err;
@@ -228,6 +252,36 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
     embed_generic_kernel<false><<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
     count_launch();
     return cudaGetLastError();
+}
+
+// The synchronous form of step 2 (Sec. 2.2 step 2: the updates are repeated k
+// times): H^0 = 0 and H^r_v = g(sum_u f([H^(r-1)_u || x_u])) for every node at
+// once. One launch per round over all (node, state) rows, the nodes of a state
+// slice spread over several blocks; messages alternate between two buffers per
+// direction (msg[2 * dir], msg[2 * dir + 1]).
+cudaError_t launch_embed_rounds(const EmbedArgs &a, const DeviceInfo &di, int rounds, float *const msg[4],
+                                cudaStream_t stream) {
+    GenericPlan p = base_plan(a, di);
+    // enough blocks per direction to fill the device about four times over
+    p.node_splits = std::max(1, std::min(a.n, (4 * di.sm_count + p.n_slices - 1) / p.n_slices));
+    p.level_begin = 0;
+    p.level_end = 1;
+    auto kern = embed_generic_kernel<false>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (err != cudaSuccess) return err;
+    dim3 grid(p.n_slices * p.node_splits, 2);
+    for (int r = 0; r <= rounds; ++r) {
+        p.round_mode = r == 0 ? 2 : 1;
+        for (int dir = 0; dir < 2; ++dir) {
+            p.M_in[dir] = msg[2 * dir + ((r + 1) & 1)];
+            p.M_out[dir] = msg[2 * dir + (r & 1)];
+        }
+        kern<<<grid, kThreads, p.smem_bytes, stream>>>(a, p);
+        count_launch();
+        err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace placeto

@@ -130,6 +130,11 @@ cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream
 cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,
                                  cudaStream_t stream);
 
+// the synchronous k-round form of step 2 on the generic kernel (rounds + 1 launches);
+// msg: four [n][B][d] buffers, two per direction
+cudaError_t launch_embed_rounds(const EmbedArgs &a, const DeviceInfo &di, int rounds, float *const msg[4],
+                                cudaStream_t stream);
+
 // embed_d32.cu: specialised message passing for d = 32 with two-layer ReLU
 // networks of hidden width 32; returns cudaErrorNotSupported when the shapes or
 // the shared-memory budget do not fit (the caller then uses the generic kernel).

@@ -292,6 +292,53 @@ def test_schedules_agree():
         compare(cfg, o, ref)
 
 
+# ------------------------------------------------- synchronous k rounds ---
+
+@pytest.mark.parametrize("d,m,layers", [(8, 3, 2), (32, 4, 2), (32, 4, 1), (64, 8, 2)])
+def test_synchronous_rounds_against_the_checker(d, m, layers):
+    """placeto_embed_rounds: H^0 = 0, every node updated at once from the
+    previous round, k rounds (the form Sec. 2.2 step 2 states)."""
+    r = rng(31 * d + layers)
+    n, B = 22, 13
+    src, dst = random_dag(r, n, 0.15)
+    F = m + 4
+    cost, nbytes = states.node_costs(r, n, normalise=True)
+    devs, cur, placed = states.random_states(r, n, m, B)
+    weights = states.policy_weights(r, d, F, m, layers, 0, 0.1)
+    g = placeto.Graph(n, src, dst)
+    w = placeto.Weights(weights)
+    X = placeto.placeto_build_features(g, dev_t(cost), dev_t(nbytes), dev_t(devs), dev_t(cur),
+                                       dev_t(placed), m)
+    Xh = X.cpu().numpy().astype(np.float64)
+    depth = g.info()["n_levels_down"]
+    for k in (0, 1, 2, 3, depth, depth + 2):
+        Hd, Hu = placeto.placeto_embed_rounds(g, w, X, k)
+        torch.cuda.synchronize()
+        assert placeto.placeto_last_launch_count() == (k + 1 if k else 0)
+        rd, ru = oracle.embed_sync(n, src, dst, Xh, weights, k)
+        assert_close(Hd, rd, "H_down after %d rounds" % k)
+        assert_close(Hu, ru, "H_up after %d rounds" % k)
+    # from depth rounds on the synchronous form has reached the progressive sweep
+    Pd, Pu = placeto.placeto_embed_forward(g, w, X)
+    torch.cuda.synchronize()
+    assert_close(Hd, Pd.cpu().numpy().astype(np.float64), "rounds vs sweep, down")
+    assert_close(Hu, Pu.cpu().numpy().astype(np.float64), "rounds vs sweep, up")
+
+
+def test_synchronous_rounds_on_the_inception_shaped_graph():
+    cfg = configs.make("inception", B=40, normalise=True)
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    X = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]),
+                                       dev_t(cfg["cur"]), dev_t(cfg["placed"]), cfg["m"])
+    Hd, Hu = placeto.placeto_embed_rounds(g, w, X, 3)
+    torch.cuda.synchronize()
+    rd, ru = oracle.embed_sync(cfg["n"], cfg["src"], cfg["dst"], X.cpu().numpy().astype(np.float64),
+                               cfg["weights"], 3)
+    assert_close(Hd, rd, "H_down")
+    assert_close(Hu, ru, "H_up")
+
+
 # ------------------------------------------------ fused and host variants ---
 
 def test_policy_forward_and_host_variant_match_the_separate_calls():
