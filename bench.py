@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--flags", type=int, default=0, help="schedule flags of placeto.h")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0)
+    ap.add_argument("--rounds", type=int, default=0,
+                    help="K > 0: the message-passing launch timed alone (roofline) is placeto_embed_rounds "
+                         "with K synchronous rounds instead of the progressive sweep")
     ap.add_argument("--episodes", type=int, default=0,
                     help="E > 0: a step is one placeto_episode_rollout call of E sampled episodes over the "
                          "workload's graph (|V| policy evaluations per episode, transitions on the device)")
@@ -359,7 +362,12 @@ def run_b200(args):
     Hd = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
     Hu = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
 
+    ws_rounds = placeto.workspace(g, w, B, placeto.CALL_EMBED_ROUNDS) if args.rounds > 0 else None
+
     def embed_only():
+        if args.rounds > 0:
+            placeto.placeto_embed_rounds(g, w, X, args.rounds, Hd, Hu, ws_rounds, stream)
+            return
         placeto.placeto_embed_forward(g, w, X, Hd, Hu, ws, args.flags, stream)
 
     def pool_only():
@@ -389,9 +397,11 @@ def run_b200(args):
         hbm_peak = float(json.load(open(peaks_path)).get("hbm_gbs", hbm_peak))
         hbm_src = "measured (MEASURED_PEAKS.json)"
     peak_tflops = sm_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
-    achieved = flops_embed(cfg) / (embed_ms * 1e-3) / 1e12
+    achieved = flops_embed(cfg) * max(1, args.rounds) / (embed_ms * 1e-3) / 1e12
     traffic, traffic_from = measured_traffic(cfg["name"])
-    roofline = {"bound": "alu", "kernel": "message passing (embed_forward, %d launch(es))" % embed_launches,
+    roofline = {"bound": "alu",
+                "kernel": ("message passing (embed_rounds, %d synchronous rounds, %d launches)" % (args.rounds, embed_launches)
+                           if args.rounds > 0 else "message passing (embed_forward, %d launch(es))" % embed_launches),
                 "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved / peak_tflops,
                 "traffic": traffic, "traffic_source": traffic_from,
                 "arithmetic": ("fp32 accumulate on mma.sync, TF32 head+tail operands (3 products)"

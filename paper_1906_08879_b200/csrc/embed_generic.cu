@@ -261,6 +261,10 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
 // direction (msg[2 * dir], msg[2 * dir + 1]).
 cudaError_t launch_embed_rounds(const EmbedArgs &a, const DeviceInfo &di, int rounds, float *const msg[4],
                                 cudaStream_t stream) {
+    if (embed_d32_applicable(a)) {
+        const cudaError_t e = launch_embed_rounds_d32(a, di, rounds, msg, stream);
+        if (e != cudaErrorNotSupported) return e;
+    }
     GenericPlan p = base_plan(a, di);
     // enough blocks per direction to fill the device about four times over
     p.node_splits = std::max(1, std::min(a.n, (4 * di.sm_count + p.n_slices - 1) / p.n_slices));

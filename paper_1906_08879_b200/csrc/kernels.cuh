@@ -135,6 +135,10 @@ cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsig
 cudaError_t launch_embed_rounds(const EmbedArgs &a, const DeviceInfo &di, int rounds, float *const msg[4],
                                 cudaStream_t stream);
 
+// embed_rounds_d32.cu: the same rounds for the shapes of embed_d32_applicable (throughput kernel)
+cudaError_t launch_embed_rounds_d32(const EmbedArgs &a, const DeviceInfo &di, int rounds,
+                                    float *const msg[4], cudaStream_t stream);
+
 // embed_d32.cu: specialised message passing for d = 32 with two-layer ReLU
 // networks of hidden width 32; returns cudaErrorNotSupported when the shapes or
 // the shared-memory budget do not fit (the caller then uses the generic kernel).
