@@ -8,9 +8,10 @@
 //     direction in registers (32 + 32 + (32 + F) + 32 values), so a warp carries
 //     a row (node, state) through gather -> g1 -> g2 -> f1 -> f2 on its own.
 //     Between layers the 32 outputs are exchanged through a per-warp shared
-//     buffer and read back as broadcast 128-bit loads: 4 FMAs per shared load.
+//     buffer and read back as broadcast 128-bit loads: 4 FMAs per shared load,
+//     issued as two packed fma.rn.f32x2 against weights kept in register pairs.
 //   - Two states of a node are in flight per warp (one on narrow levels), with
-//     four accumulators per row, for instruction-level parallelism.
+//     four dependent accumulator chains per row.
 //   - Messages never leave the SM: m_u lives in a shared-memory slot from the
 //     level of u until its last consumer's level (slots assigned on the host).
 //     Global traffic is the compulsory part only: read x, write h.
@@ -39,35 +40,57 @@ struct D32Plan {
     size_t smem_bytes;
 };
 
+typedef unsigned long long pair_t;   // two FP32 values in one 64-bit register pair
+
+__device__ __forceinline__ pair_t pack2(float lo, float hi) {
+    pair_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(pair_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// Two independent FP32 FMAs in one instruction (sm_100 packed arithmetic): half
+// the FMA issue slots, the same rounding as two fmaf.
+__device__ __forceinline__ pair_t fma2(pair_t a, pair_t b, pair_t c) {
+    pair_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // out[r] = bias + in[r] . w for R rows whose K inputs are read as broadcast
-// float4 from shared memory; four independent accumulators per row keep the
-// FMA pipe busy without lengthening the dependent chain.
+// 128-bit loads from shared memory. The weights are kept as pairs (w[2i],
+// w[2i + 1]) so that every load feeds two packed FMAs; two pair accumulators per
+// row, i.e. four dependent chains of K / 4 FMAs.
 template <int R, int K>
-__device__ __forceinline__ void matvec(const float (&w)[K], float bias, const float *in,
+__device__ __forceinline__ void matvec(const pair_t (&w)[K / 2], float bias, const float *in,
                                        int row_stride, float (&out)[R]) {
-    float acc[R][2];
+    pair_t acc[R][2];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        acc[r][0] = bias;
-        acc[r][1] = 0.f;
+        acc[r][0] = pack2(bias, 0.f);
+        acc[r][1] = 0ull;
     }
 #pragma unroll
     for (int k = 0; k < K; k += 4) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const float4 u = *reinterpret_cast<const float4 *>(in + r * row_stride + k);
-            acc[r][0] = fmaf(u.x, w[k], acc[r][0]);
-            acc[r][1] = fmaf(u.y, w[k + 1], acc[r][1]);
-            acc[r][0] = fmaf(u.z, w[k + 2], acc[r][0]);
-            acc[r][1] = fmaf(u.w, w[k + 3], acc[r][1]);
+            const ulonglong2 u = *reinterpret_cast<const ulonglong2 *>(in + r * row_stride + k);
+            acc[r][0] = fma2(u.x, w[k / 2], acc[r][0]);
+            acc[r][1] = fma2(u.y, w[k / 2 + 1], acc[r][1]);
         }
     }
 #pragma unroll
-    for (int r = 0; r < R; ++r) out[r] = acc[r][0] + acc[r][1];
+    for (int r = 0; r < R; ++r) {
+        float a, b, c, d;
+        unpack2(acc[r][0], a, b);
+        unpack2(acc[r][1], c, d);
+        out[r] = (a + b) + (c + d);
+    }
 }
 
 struct Weights32 {
-    float g1[kD], g2[kD], f2[kD];
+    pair_t g1[kD / 2], g2[kD / 2], f2[kD / 2];   // column `lane`, rows in pairs
     float bg1, bg2, bf1, bf2;
 };
 
@@ -77,7 +100,7 @@ struct Weights32 {
 // schedule lookups are done once. A, Bf: the warp's exchange buffers, R rows of
 // KF floats each. All shared-memory offsets are 32-bit.
 template <int R, int KF>
-__device__ __forceinline__ void run_node(const Weights32 &w, const float (&wf1)[KF], int pos,
+__device__ __forceinline__ void run_node(const Weights32 &w, const pair_t (&wf1)[KF / 2], int pos,
                                          int q, int s0, bool last_live, int nb, int S, int F,
                                          int lane, const int4 *meta, const int *nbr_slot,
                                          float *msg, const float *xs, float *__restrict__ H,
@@ -193,15 +216,17 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     // ---- this lane's weight columns
     const DevMlp f = a.f[dir], g = a.g[dir];
     Weights32 w;
-    float wf1[KF];
+    pair_t wf1[KF / 2];
 #pragma unroll
-    for (int k = 0; k < kD; ++k) {
-        w.g1[k] = g.W1[k * kD + lane];
-        w.g2[k] = g.W2[k * kD + lane];
-        w.f2[k] = f.W2[k * kD + lane];
+    for (int k = 0; k < kD; k += 2) {
+        w.g1[k / 2] = pack2(g.W1[k * kD + lane], g.W1[(k + 1) * kD + lane]);
+        w.g2[k / 2] = pack2(g.W2[k * kD + lane], g.W2[(k + 1) * kD + lane]);
+        w.f2[k / 2] = pack2(f.W2[k * kD + lane], f.W2[(k + 1) * kD + lane]);
     }
 #pragma unroll
-    for (int k = 0; k < KF; ++k) wf1[k] = (k < kD + F) ? f.W1[k * kD + lane] : 0.f;
+    for (int k = 0; k < KF; k += 2)
+        wf1[k / 2] = pack2(k < kD + F ? f.W1[k * kD + lane] : 0.f,
+                           k + 1 < kD + F ? f.W1[(k + 1) * kD + lane] : 0.f);
     w.bg1 = g.b1[lane]; w.bg2 = g.b2[lane]; w.bf1 = f.b1[lane]; w.bf2 = f.b2[lane];
     const float *__restrict__ X = a.X;
     float *__restrict__ H = a.H[dir];
