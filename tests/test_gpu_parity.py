@@ -339,6 +339,26 @@ def test_synchronous_rounds_on_the_inception_shaped_graph():
     assert_close(Hu, ru, "H_up")
 
 
+def test_simple_partitioner_variant_is_the_pooling_on_zero_embeddings():
+    """The paper's "simple partitioner" ablation (Sec. 4, alternative policy
+    architectures) pools the raw features of the three sets without the message
+    passing: placeto_policy_logits on zero embeddings."""
+    cfg = configs.make("inception", B=24, normalise=True)
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    cur = dev_t(cfg["cur"])
+    X = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]),
+                                       cur, dev_t(cfg["placed"]), cfg["m"])
+    Z = torch.zeros((cfg["n"], 24, cfg["d"]), dtype=torch.float32, device="cuda")
+    logits, probs = placeto.placeto_policy_logits(g, w, X, Z, Z, cur)
+    torch.cuda.synchronize()
+    zeros = np.zeros((cfg["n"], 24, cfg["d"]))
+    rl, rp = oracle.policy(cfg["n"], cfg["src"], cfg["dst"], X.cpu().numpy().astype(np.float64), zeros,
+                           zeros, cfg["cur"], cfg["weights"])
+    assert_close(logits, rl, "logits")
+    assert_argmax(logits, rl)
+
+
 # ------------------------------------------------ fused and host variants ---
 
 def test_policy_forward_and_host_variant_match_the_separate_calls():
