@@ -290,6 +290,31 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
                                        void *stream);
 
 /*
+ * Simulated run time of P placements of the graph under the event-based execution
+ * model of the paper's simulator (Appendix A.4): one operation at a time per
+ * device, taken from a FIFO queue of runnable operations; one output tensor at a
+ * time per device bus, overlapping with compute; an operation becomes runnable when
+ * all parents have finished and their outputs have arrived on its device; an
+ * operation takes cost[v], a transfer bytes[u] / bandwidth; the result is the time
+ * stamp of the last operation to finish. One thread simulates one placement.
+ * Readings where the paper is silent: one run time per operation whatever the
+ * device; a tensor is sent once to each distinct device that hosts a child; a free
+ * device or bus starts the head of its queue at once; equal time stamps are handled
+ * in the order the events were created; peak memory is not modelled.
+ *
+ * cost, bytes : DEVICE float[n].          dev : DEVICE uint8[P][n], devices < m.
+ * bandwidth   : > 0, in units of bytes[] per unit of cost[].
+ * runtime     : DEVICE double[P]; NaN for a placement that names a device >= m.
+ * workspace   : DEVICE, at least placeto_simulator_workspace_bytes(g, P, m).
+ * Times are IEEE doubles added and divided in the model's order: reproducible.
+ */
+size_t placeto_simulator_workspace_bytes(const placeto_graph *g, int32_t P, int32_t m);
+placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cost, const float *bytes,
+                                        const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
+                                        double *runtime, void *workspace, size_t workspace_bytes,
+                                        void *stream);
+
+/*
  * placeto_policy_logits without a workspace argument, for callers that must not
  * allocate device memory. (The paper has no counterpart: this is a deployment
  * variant of the call above, not a step of the method.)

@@ -28,7 +28,8 @@ EXPORTS = (
     "placeto_graph_host_view", "placeto_graph_destroy", "placeto_workspace_bytes",
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
-    "placeto_episode_rollout", "placeto_embed_rounds", "placeto_last_launch_count",
+    "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulator_workspace_bytes", "placeto_simulate_runtime",
+    "placeto_last_launch_count",
 )
 
 
@@ -72,10 +73,11 @@ def _load() -> ctypes.CDLL:
     lib.placeto_graph_destroy.argtypes = [ctypes.c_void_p]
     lib.placeto_workspace_bytes.restype = ctypes.c_size_t
     lib.placeto_last_launch_count.restype = ctypes.c_int32
+    lib.placeto_simulator_workspace_bytes.restype = ctypes.c_size_t
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
-                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds"):
+                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -347,6 +349,24 @@ def placeto_episode_rollout(g: Graph, w: Weights, cost, nbytes, order, dev, unif
                                         ctypes.c_uint32(flags), _stream(stream)),
            "placeto_episode_rollout")
     return dev, actions, logp
+
+
+def placeto_simulate_runtime(g: Graph, cost, nbytes, dev, m: int, bandwidth: float, runtime=None,
+                             ws=None, stream=None):
+    """Simulated run time (float64 [P]) of the P placements in `dev` (uint8 [P][n])."""
+    P = dev.shape[0]
+    if runtime is None:
+        runtime = torch.empty((P,), dtype=torch.float64, device=dev.device)
+    if ws is None:
+        need = int(_lib.placeto_simulator_workspace_bytes(g.handle, ctypes.c_int32(P), ctypes.c_int32(m)))
+        if need == 0:
+            raise PlacetoError(1, "placeto_simulator_workspace_bytes")
+        ws = torch.empty(need, dtype=torch.uint8, device=dev.device)
+    _check(_lib.placeto_simulate_runtime(g.handle, _p(cost), _p(nbytes), _p(dev), ctypes.c_int32(P),
+                                         ctypes.c_int32(m), ctypes.c_double(bandwidth), _p(runtime),
+                                         _p(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "placeto_simulate_runtime")
+    return runtime
 
 
 def placeto_last_launch_count() -> int:

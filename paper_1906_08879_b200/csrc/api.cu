@@ -17,6 +17,7 @@ struct placeto_graph {
     int device = -1;
     DeviceInfo info{};
     int *d_ints = nullptr;       // one allocation for all int arrays
+    int *d_child_ptr = nullptr, *d_child = nullptr, *d_n_parents = nullptr;   // inside d_ints
     uint8_t *d_relation = nullptr;
     DevLevels lv[2]{};
 };
@@ -294,6 +295,11 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
                                        p.nbr.size(), p.own_slot.size(), p.nbr_slot.size()};
         for (int k = 0; k < kArrays; ++k) { offs[dir][k] = total; total += (sizes[k] + 3) & ~size_t(3); }
     }
+    // and, by node id, the children lists and parent counts of the runtime simulator
+    const size_t sim_off[3] = {total, total + ((g->host.child_ptr.size() + 3) & ~size_t(3)),
+                               total + ((g->host.child_ptr.size() + 3) & ~size_t(3)) +
+                                   ((g->host.child.size() + 3) & ~size_t(3))};
+    total = sim_off[2] + ((g->host.n_parents.size() + 3) & ~size_t(3));
     if (cudaMalloc(&g->d_ints, std::max<size_t>(total, 4) * sizeof(int)) != cudaSuccess)
         return fail(PLACETO_ERR_NO_MEMORY);
     if (cudaMalloc(&g->d_relation, g->host.relation.size()) != cudaSuccess)
@@ -316,6 +322,17 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
         g->lv[dir].own_slot = g->d_ints + offs[dir][4];
         g->lv[dir].nbr_slot = g->d_ints + offs[dir][5];
         g->lv[dir].n_nbr = static_cast<int>(p.nbr.size());
+    }
+    {
+        const std::vector<int32_t> *vecs[3] = {&g->host.child_ptr, &g->host.child, &g->host.n_parents};
+        int **dst[3] = {&g->d_child_ptr, &g->d_child, &g->d_n_parents};
+        for (int k = 0; k < 3; ++k) {
+            *dst[k] = g->d_ints + sim_off[k];
+            if (!vecs[k]->empty() &&
+                cudaMemcpy(*dst[k], vecs[k]->data(), vecs[k]->size() * sizeof(int),
+                           cudaMemcpyHostToDevice) != cudaSuccess)
+                return fail(PLACETO_ERR_CUDA);
+        }
     }
     if (cudaMemcpy(g->d_relation, g->host.relation.data(), g->host.relation.size(),
                    cudaMemcpyHostToDevice) != cudaSuccess)
@@ -623,6 +640,34 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
         if (s == PLACETO_OK) s = cuda_status(launch_episode_step(ep, t, st));
     }
     return s;
+}
+
+size_t placeto_simulator_workspace_bytes(const placeto_graph *g, int32_t P, int32_t m) {
+    if (!g || P < 1 || m < 1 || m > PLACETO_MAX_M) return 0;
+    return sim_workspace_bytes(g->host.n, (int)g->host.n_edges, m, P);
+}
+
+placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cost, const float *bytes,
+                                        const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
+                                        double *runtime, void *workspace, size_t workspace_bytes,
+                                        void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device || P < 1 || m < 1 || m > PLACETO_MAX_M) return PLACETO_ERR_INVALID_ARG;
+    if (!(bandwidth > 0.0)) return PLACETO_ERR_INVALID_ARG;
+    if (!cost || !bytes || !dev || !runtime || !workspace) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(runtime) ||
+        !aligned16(workspace))
+        return PLACETO_ERR_INVALID_ARG;
+    if (workspace_bytes < sim_workspace_bytes(g->host.n, (int)g->host.n_edges, m, P))
+        return PLACETO_ERR_WORKSPACE;
+    SimArgs a;
+    a.n = g->host.n; a.n_edges = (int)g->host.n_edges; a.m = m; a.P = P;
+    a.child_ptr = g->d_child_ptr; a.child = g->d_child; a.n_parents = g->d_n_parents;
+    a.cost = cost; a.bytes = bytes; a.dev = dev;
+    a.bandwidth = bandwidth;
+    a.runtime = runtime;
+    a.workspace = static_cast<char *>(workspace);
+    return cuda_status(launch_simulator(a, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t placeto_last_launch_count(void) { return t_launches; }

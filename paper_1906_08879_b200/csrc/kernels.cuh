@@ -78,6 +78,16 @@ struct EpisodeArgs {
     float *X;                  // [n][E][m + 4] raw features, patched in place after every step
 };
 
+struct SimArgs {
+    int n, n_edges, m, P;
+    const int *child_ptr, *child, *n_parents;   // by node id
+    const float *cost, *bytes;                  // [n]
+    const uint8_t *dev;                         // [P][n]
+    double bandwidth;
+    double *runtime;                            // [P]
+    char *workspace;
+};
+
 struct DeviceInfo {
     int sm_count;
     int max_smem_optin;   // bytes per block
@@ -124,6 +134,10 @@ cudaError_t launch_features(int n, int B, int m, const float *cost, const float 
 // episode.cu: the MDP transition between two policy evaluations of an episode
 cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream);
 cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream);
+
+// simulator.cu: event-based run time of P placements, one thread each
+size_t sim_workspace_bytes(int n, int n_edges, int m, int P);
+cudaError_t launch_simulator(const SimArgs &a, cudaStream_t stream);
 
 // embed_generic.cu: dimension-generic message passing. schedule is one of
 // PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.

@@ -117,6 +117,14 @@ placeto_status build_plan(int32_t n, int64_t n_edges, const int32_t *src, const 
         bucket(n, level_up, chi, plan.dir[1]);
         assign_slots(n, level_down, plan.dir[0]);
         assign_slots(n, level_up, plan.dir[1]);
+        plan.child_ptr.assign(n + 1, 0);
+        plan.child.clear();
+        plan.n_parents.assign(n, 0);
+        for (int32_t v = 0; v < n; ++v) {
+            plan.child.insert(plan.child.end(), chi[v].begin(), chi[v].end());
+            plan.child_ptr[v + 1] = static_cast<int32_t>(plan.child.size());
+            plan.n_parents[v] = static_cast<int32_t>(par[v].size());
+        }
         plan.max_level_width = 0;
         for (int dir = 0; dir < 2; ++dir)
             for (int32_t l = 0; l < plan.dir[dir].n_levels; ++l)

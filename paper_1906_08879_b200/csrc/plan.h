@@ -31,6 +31,8 @@ struct HostPlan {
     int32_t max_degree = 0;          // largest neighbour set, both directions
     LevelPlan dir[2];                // 0 top-down, 1 bottom-up
     std::vector<uint8_t> relation;   // [n * n], see placeto_graph_host_view
+    // by node id, for the runtime simulator: children (ascending) and number of parents
+    std::vector<int32_t> child_ptr, child, n_parents;
 };
 
 // Validates the edge list and fills `plan`. Returns PLACETO_OK,
