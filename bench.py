@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--rounds", type=int, default=0,
                     help="K > 0: the message-passing launch timed alone (roofline) is placeto_embed_rounds "
                          "with K synchronous rounds instead of the progressive sweep")
+    ap.add_argument("--simulate", type=int, default=0,
+                    help="P > 0: instead of the policy path, time placeto_simulate_runtime on P random "
+                         "placements of the workload's graph (its own metric: simulated placements/s)")
     ap.add_argument("--episodes", type=int, default=0,
                     help="E > 0: a step is one placeto_episode_rollout call of E sampled episodes over the "
                          "workload's graph (|V| policy evaluations per episode, transitions on the device)")
@@ -438,8 +441,53 @@ def run_b200(args):
     return 0
 
 
+def run_simulator(args):
+    """Extra mode: the runtime simulator on P random placements (one JSON line, own metric)."""
+    import torch
+    import paper_1906_08879_b200 as placeto
+    from oracle import simulator
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    cfg = make_workload(args.workload)
+    n, m, P = cfg["n"], cfg["m"], args.simulate
+    rng = np.random.Generator(np.random.PCG64(99))
+    devs_h = rng.integers(0, m, size=(P, n)).astype(np.uint8)
+    g = placeto.Graph(n, cfg["src"], cfg["dst"])
+    dev_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    cost, nbytes, devs = dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(devs_h)
+    out = torch.empty((P,), dtype=torch.float64, device="cuda")
+    bw = 1e4
+    need = int(placeto.binding._lib.placeto_simulator_workspace_bytes(g.handle, P, m))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        placeto.placeto_simulate_runtime(g, cost, nbytes, devs, m, bw, out, ws, stream)
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record(stream)
+    for _ in range(args.steps):
+        placeto.placeto_simulate_runtime(g, cost, nbytes, devs, m, bw, out, ws, stream)
+    e.record(stream)
+    torch.cuda.synchronize()
+    ms = s.elapsed_time(e) / args.steps
+    k = min(P, 32)
+    t0 = time.perf_counter()
+    ref = simulator.runtimes(n, cfg["src"], cfg["dst"], cfg["cost"], cfg["bytes"], devs_h[:k], m, bw)
+    cpu_s = time.perf_counter() - t0
+    assert np.array_equal(out.cpu().numpy()[:k], ref), "simulator disagrees with the CPU checker"
+    print(json.dumps({"metric": "simulated placements/sec (event-based runtime simulator)",
+                      "value": P / (ms * 1e-3), "unit": "placements/s", "n_gpus": 1, "steps": args.steps,
+                      "ms_per_step": ms, "higher_is_better": True, "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": cfg["name"] + "-simulator", "n_nodes": n, "placements": P,
+                                 "devices": m, "bandwidth": bw},
+                      "cpu_baseline": {"value": k / cpu_s, "unit": "placements/s", "cores": 1, "kind": "oracle",
+                                       "sample": "%d placements, pure-Python event loop" % k}}))
+    return 0
+
+
 def main():
     args = parse_args()
+    if args.simulate > 0 and args.impl != "reference":
+        return run_simulator(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_b200(args)
