@@ -168,7 +168,8 @@ typedef enum {
     PLACETO_CALL_FORWARD = 2,     /* placeto_policy_forward */
     PLACETO_CALL_FORWARD_HOST = 3,/* placeto_policy_forward_host */
     PLACETO_CALL_EPISODE = 4,     /* placeto_episode_rollout (B = number of episodes) */
-    PLACETO_CALL_EMBED_ROUNDS = 5 /* placeto_embed_rounds */
+    PLACETO_CALL_EMBED_ROUNDS = 5,/* placeto_embed_rounds */
+    PLACETO_CALL_GRADIENT = 6     /* placeto_policy_gradient */
 } placeto_call;
 
 /* Bytes of DEVICE workspace `call` needs for batch size B (0 on invalid arguments).
@@ -313,6 +314,35 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
                                         const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
                                         double *runtime, void *workspace, size_t workspace_bytes,
                                         void *stream);
+
+/*
+ * Gradient of the training objective with respect to every weight and bias of the
+ * policy, for a batch of B states (Appendix A.1 of the paper: REINFORCE,
+ * sum_b grad log pi(a_b | s_b) * A_b with A_b = return minus baseline; Appendix A.6:
+ * an entropy term that encourages exploration):
+ *     J = sum_b advantages[b] * log pi(actions[b] | s_b) + beta * sum_b H(pi(. | s_b)),
+ *     H(p) = - sum_k p_k log p_k.
+ * Reverse-mode differentiation of the forward path: the head and the pooling per
+ * state, the two message-passing sweeps level by level in reverse, then every
+ * layer's dW = in^T dpre, db = sum dpre as chunked sums added in a fixed order (no
+ * atomics: reproducible bit for bit).
+ *
+ * X, H_down, H_up : DEVICE, as produced by placeto_build_features / placeto_embed_forward
+ *                   for the same states and weights.
+ * cur, actions    : DEVICE int32[B] (actions < m; a state whose cur is outside [0, n)
+ *                   contributes nothing).      advantages : DEVICE float[B].
+ * grads           : a placeto_weights of the same shapes as w whose pointers address
+ *                   writable DEVICE buffers; every array is overwritten with dJ/d(array).
+ * workspace       : DEVICE, at least placeto_workspace_bytes(.., PLACETO_CALL_GRADIENT, 0):
+ *                   about 2 * n * B * (2 * (hidden_f + hidden_g) + 6 d) + 3 n B d floats.
+ * Shapes: two-layer ReLU f and g, single-layer ReLU l_i and h_i, two-layer head with a
+ * ReLU hidden layer and a linear output; otherwise PLACETO_ERR_UNSUPPORTED.
+ */
+placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_weights *w, const float *X,
+                                       const float *H_down, const float *H_up, const int32_t *cur,
+                                       const int32_t *actions, const float *advantages, float beta,
+                                       int32_t B, const placeto_weights *grads, void *workspace,
+                                       size_t workspace_bytes, void *stream);
 
 /*
  * placeto_policy_logits without a workspace argument, for callers that must not

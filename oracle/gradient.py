@@ -121,7 +121,9 @@ def gradient(cfg, actions, advantages, beta=0.0):
     J = objective(logp, actions, advantages, beta)
     J.backward()
     def grads(net):
-        return {k: v.grad.numpy().copy() for k, v in net.items()}
+        # an array the objective does not depend on (f on a graph without edges) has no .grad: zero
+        return {k: (v.grad.numpy().copy() if v.grad is not None else np.zeros(tuple(v.shape)))
+                for k, v in net.items()}
     out = {k: grads(t[k]) for k in NETS}
     for k in SETS:
         out[k] = [grads(x) for x in t[k]]

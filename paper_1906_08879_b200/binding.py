@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libplaceto.so")
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
 PLACETO_FMA_ONLY, PLACETO_TENSOR = 16, 32
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
-CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE, CALL_EMBED_ROUNDS = 0, 1, 2, 3, 4, 5
+CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE, CALL_EMBED_ROUNDS, CALL_GRADIENT = 0, 1, 2, 3, 4, 5, 6
 
 EXPORTS = (
     "placeto_status_string", "placeto_graph_create", "placeto_graph_info",
@@ -29,7 +29,7 @@ EXPORTS = (
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
     "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulator_workspace_bytes", "placeto_simulate_runtime",
-    "placeto_last_launch_count",
+    "placeto_policy_gradient", "placeto_last_launch_count",
 )
 
 
@@ -77,7 +77,7 @@ def _load() -> ctypes.CDLL:
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
-                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime"):
+                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime", "placeto_policy_gradient"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -183,19 +183,20 @@ class Weights:
     def __init__(self, weights: dict, device="cuda"):
         self.d, self.F, self.m = int(weights["d"]), int(weights["F"]), int(weights["m"])
         self._keep = []
+        self.tensors = {}            # (net name, index or None, array name) -> device tensor
         self.c = _Weights()
         self.c.d, self.c.F, self.c.m = self.d, self.F, self.m
         dev = torch.device(device)
         for name in ("f_down", "g_down", "f_up", "g_up", "head"):
             if name in weights:
-                setattr(self.c, name, self._mlp(weights[name], dev))
+                setattr(self.c, name, self._mlp(weights[name], dev, (name, None)))
         for name in ("l", "h"):
             if name in weights:
                 arr = getattr(self.c, name)
                 for i in range(3):
-                    arr[i] = self._mlp(weights[name][i], dev)
+                    arr[i] = self._mlp(weights[name][i], dev, (name, i))
 
-    def _mlp(self, net: dict, dev) -> _Mlp:
+    def _mlp(self, net: dict, dev, where=None) -> _Mlp:
         ptr = {}
         for k in ("W1", "b1", "W2", "b2"):
             a = net.get(k)
@@ -204,6 +205,8 @@ class Weights:
                 continue
             t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev)
             self._keep.append(t)
+            if where is not None:
+                self.tensors[where + (k,)] = t
             ptr[k] = t.data_ptr()
         return _Mlp(net["n_layers"], net["in_dim"], net.get("hidden_dim", net["out_dim"]),
                     net["out_dim"], ptr["W1"], ptr["b1"], ptr["W2"], ptr["b2"],
@@ -367,6 +370,36 @@ def placeto_simulate_runtime(g: Graph, cost, nbytes, dev, m: int, bandwidth: flo
                                          _p(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
            "placeto_simulate_runtime")
     return runtime
+
+
+def zero_gradients(weights: dict, device="cuda") -> "Weights":
+    """A Weights object of the same shapes filled with zeros (gradient buffers)."""
+    def z(net):
+        out = dict(net)
+        for k in ("W1", "b1", "W2", "b2"):
+            if net.get(k) is not None:
+                out[k] = np.zeros_like(np.asarray(net[k], dtype=np.float32))
+        return out
+    g = {k: weights[k] for k in ("d", "F", "m")}
+    for k in ("f_down", "g_down", "f_up", "g_up", "head"):
+        g[k] = z(weights[k])
+    for k in ("l", "h"):
+        g[k] = [z(x) for x in weights[k]]
+    return Weights(g, device)
+
+
+def placeto_policy_gradient(g: Graph, w: Weights, X, H_down, H_up, cur, actions, advantages,
+                            beta: float, grads: Weights, ws=None, stream=None):
+    """dJ/d(weights) into `grads` (a Weights of the same shapes, see zero_gradients)."""
+    B = X.shape[1]
+    if ws is None:
+        ws = workspace(g, w, B, CALL_GRADIENT, 0, X.device)
+    _check(_lib.placeto_policy_gradient(g.handle, ctypes.byref(w.c), _p(X), _p(H_down), _p(H_up), _p(cur),
+                                        _p(actions), _p(advantages), ctypes.c_float(beta),
+                                        ctypes.c_int32(B), ctypes.byref(grads.c), _p(ws),
+                                        ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "placeto_policy_gradient")
+    return grads
 
 
 def placeto_last_launch_count() -> int:

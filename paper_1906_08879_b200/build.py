@@ -19,7 +19,7 @@ LIB = os.path.join(HERE, "libplaceto.so")
 
 SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "embed_d32.cu", "embed_d64.cu", "embed_mma.cu",
            "policy_generic.cu", "policy_d32.cu", "policy_d64.cu", "episode.cu",
-           "embed_rounds_d32.cu", "simulator.cu"]
+           "embed_rounds_d32.cu", "simulator.cu", "gradient.cu"]
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo",
               "-gencode", "arch=compute_100a,code=sm_100a",

@@ -18,6 +18,7 @@ struct placeto_graph {
     DeviceInfo info{};
     int *d_ints = nullptr;       // one allocation for all int arrays
     int *d_child_ptr = nullptr, *d_child = nullptr, *d_n_parents = nullptr;   // inside d_ints
+    int *d_parent_ptr = nullptr, *d_parent = nullptr;                          // inside d_ints
     uint8_t *d_relation = nullptr;
     DevLevels lv[2]{};
 };
@@ -93,6 +94,13 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE)) {
         L.msg[0] = take(n * B * d * sizeof(float));
         L.msg[1] = take(n * B * d * sizeof(float));
+    }
+    if (call == PLACETO_CALL_GRADIENT) {
+        const int Hf = std::max(w->f_down.hidden_dim, w->f_up.hidden_dim);
+        const int Hg = std::max(w->g_down.hidden_dim, w->g_up.hidden_dim);
+        L.total = policy_gradient_workspace_floats((int)n, B, w->d, w->F, w->m, Hf, Hg, w->head.hidden_dim) *
+                  sizeof(float);
+        return L;
     }
     if (call == PLACETO_CALL_EMBED_ROUNDS) {
         L.msg_alt[0] = take(n * B * d * sizeof(float));
@@ -295,11 +303,11 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
                                        p.nbr.size(), p.own_slot.size(), p.nbr_slot.size()};
         for (int k = 0; k < kArrays; ++k) { offs[dir][k] = total; total += (sizes[k] + 3) & ~size_t(3); }
     }
-    // and, by node id, the children lists and parent counts of the runtime simulator
-    const size_t sim_off[3] = {total, total + ((g->host.child_ptr.size() + 3) & ~size_t(3)),
-                               total + ((g->host.child_ptr.size() + 3) & ~size_t(3)) +
-                                   ((g->host.child.size() + 3) & ~size_t(3))};
-    total = sim_off[2] + ((g->host.n_parents.size() + 3) & ~size_t(3));
+    // and, by node id: children, parent counts (runtime simulator), parents (policy gradient)
+    const std::vector<int32_t> *extra[5] = {&g->host.child_ptr, &g->host.child, &g->host.n_parents,
+                                            &g->host.parent_ptr, &g->host.parent};
+    size_t sim_off[5];
+    for (int k = 0; k < 5; ++k) { sim_off[k] = total; total += (extra[k]->size() + 3) & ~size_t(3); }
     if (cudaMalloc(&g->d_ints, std::max<size_t>(total, 4) * sizeof(int)) != cudaSuccess)
         return fail(PLACETO_ERR_NO_MEMORY);
     if (cudaMalloc(&g->d_relation, g->host.relation.size()) != cudaSuccess)
@@ -324,12 +332,11 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
         g->lv[dir].n_nbr = static_cast<int>(p.nbr.size());
     }
     {
-        const std::vector<int32_t> *vecs[3] = {&g->host.child_ptr, &g->host.child, &g->host.n_parents};
-        int **dst[3] = {&g->d_child_ptr, &g->d_child, &g->d_n_parents};
-        for (int k = 0; k < 3; ++k) {
+        int **dst[5] = {&g->d_child_ptr, &g->d_child, &g->d_n_parents, &g->d_parent_ptr, &g->d_parent};
+        for (int k = 0; k < 5; ++k) {
             *dst[k] = g->d_ints + sim_off[k];
-            if (!vecs[k]->empty() &&
-                cudaMemcpy(*dst[k], vecs[k]->data(), vecs[k]->size() * sizeof(int),
+            if (!extra[k]->empty() &&
+                cudaMemcpy(*dst[k], extra[k]->data(), extra[k]->size() * sizeof(int),
                            cudaMemcpyHostToDevice) != cudaSuccess)
                 return fail(PLACETO_ERR_CUDA);
         }
@@ -390,7 +397,9 @@ void placeto_graph_destroy(placeto_graph *g) {
 size_t placeto_workspace_bytes(const placeto_graph *g, const placeto_weights *w, int32_t B,
                                placeto_call call, uint32_t flags) {
     if (!g || !w || B < 1 || !flags_ok(flags) || dims_ok(w) != PLACETO_OK) return 0;
-    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_EMBED_ROUNDS) return 0;
+    if (call < PLACETO_CALL_EMBED || call > PLACETO_CALL_GRADIENT) return 0;
+    if (call == PLACETO_CALL_GRADIENT && (embed_weights_ok(w) != PLACETO_OK || pool_weights_ok(w) != PLACETO_OK))
+        return 0;
     placeto_graph tmp_info;   // HOST_ONLY graphs have no device info: assume a full B200
     const placeto_graph *use = g;
     if (!g->on_device) {
@@ -668,6 +677,67 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
     a.runtime = runtime;
     a.workspace = static_cast<char *>(workspace);
     return cuda_status(launch_simulator(a, static_cast<cudaStream_t>(stream)));
+}
+
+placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_weights *w, const float *X,
+                                       const float *H_down, const float *H_up, const int32_t *cur,
+                                       const int32_t *actions, const float *advantages, float beta,
+                                       int32_t B, const placeto_weights *grads, void *workspace,
+                                       size_t workspace_bytes, void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    placeto_status s = embed_weights_ok(w);
+    if (s == PLACETO_OK) s = pool_weights_ok(w);
+    if (s != PLACETO_OK) return s;
+    if (B < 1 || !grads) return PLACETO_ERR_INVALID_ARG;
+    // the gradient buffers mirror the weights' shapes
+    if (grads->d != w->d || grads->F != w->F || grads->m != w->m) return PLACETO_ERR_INVALID_ARG;
+    const placeto_mlp *wn[11] = {&w->f_down, &w->f_up, &w->g_down, &w->g_up, &w->l[0], &w->l[1], &w->l[2],
+                                 &w->h[0], &w->h[1], &w->h[2], &w->head};
+    const placeto_mlp *gn[11] = {&grads->f_down, &grads->f_up, &grads->g_down, &grads->g_up, &grads->l[0],
+                                 &grads->l[1], &grads->l[2], &grads->h[0], &grads->h[1], &grads->h[2],
+                                 &grads->head};
+    for (int i = 0; i < 11; ++i) {
+        if (gn[i]->n_layers != wn[i]->n_layers || gn[i]->in_dim != wn[i]->in_dim ||
+            gn[i]->out_dim != wn[i]->out_dim ||
+            (wn[i]->n_layers == 2 && gn[i]->hidden_dim != wn[i]->hidden_dim))
+            return PLACETO_ERR_INVALID_ARG;
+        if (!gn[i]->W1 || !gn[i]->b1 || !aligned16(gn[i]->W1) || !aligned16(gn[i]->b1)) return PLACETO_ERR_INVALID_ARG;
+        if (wn[i]->n_layers == 2 && (!gn[i]->W2 || !gn[i]->b2 || !aligned16(gn[i]->W2) || !aligned16(gn[i]->b2)))
+            return PLACETO_ERR_INVALID_ARG;
+    }
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_GRADIENT);
+    s = common_checks(g, B, workspace, workspace_bytes, L.total, 0);
+    if (s != PLACETO_OK) return s;
+    if (!X || !H_down || !H_up || !cur || !actions || !advantages) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(H_down) || !aligned16(H_up) || !aligned16(cur) ||
+        !aligned16(actions) || !aligned16(advantages))
+        return PLACETO_ERR_INVALID_ARG;
+    GradArgs a{};
+    a.n = g->host.n; a.B = B; a.d = w->d; a.F = w->F; a.m = w->m;
+    a.relation = g->d_relation;
+    a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
+    a.child_ptr = g->d_child_ptr; a.child = g->d_child;
+    a.parent_ptr = g->d_parent_ptr; a.parent = g->d_parent;
+    a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
+    a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
+    for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
+    a.head = to_dev(w->head);
+    if (!policy_gradient_applicable(a)) return PLACETO_ERR_UNSUPPORTED;
+    a.X = X; a.H[0] = H_down; a.H[1] = H_up;
+    a.cur = cur; a.actions = actions; a.advantages = advantages; a.beta = beta;
+    auto out = [](const placeto_mlp &m) {
+        GradOut o;
+        o.W1 = const_cast<float *>(m.W1); o.b1 = const_cast<float *>(m.b1);
+        o.W2 = const_cast<float *>(m.W2); o.b2 = const_cast<float *>(m.b2);
+        return o;
+    };
+    a.gf[0] = out(grads->f_down); a.gf[1] = out(grads->f_up);
+    a.gg[0] = out(grads->g_down); a.gg[1] = out(grads->g_up);
+    for (int i = 0; i < 3; ++i) { a.gl[i] = out(grads->l[i]); a.gh[i] = out(grads->h[i]); }
+    a.ghead = out(grads->head);
+    return cuda_status(launch_policy_gradient(a, g->info, static_cast<float *>(workspace),
+                                              static_cast<cudaStream_t>(stream)));
 }
 
 int32_t placeto_last_launch_count(void) { return t_launches; }

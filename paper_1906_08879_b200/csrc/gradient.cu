@@ -1,0 +1,552 @@
+// Gradient of the policy objective with respect to every weight (Appendix A.1
+// and A.6 of the Placeto paper: the REINFORCE term sum_b A_b log pi(a_b | s_b)
+// plus an entropy term beta sum_b H(pi(. | s_b))), by reverse-mode
+// differentiation of the forward path:
+//
+//   1. messages   : for every (node, state) row the hidden layer and the output of
+//                   f are recomputed from H and X and stored (both directions);
+//   2. head/pool  : per state, the pooled sums, h_i, the head and the softmax are
+//                   recomputed, d(objective)/d(logits) is formed and pushed back
+//                   through the head, h_i and l_i down to d/d(e_u) of every node;
+//   3. sweeps     : per direction, levels in reverse order, d/d(h_v) is pushed
+//                   through g to the summed messages and through f to the
+//                   neighbours' embeddings (a node gathers from its consumers:
+//                   no scattered adds);
+//   4. weights    : each network layer's dW = in^T dpre and db = sum dpre over the
+//                   stored per-row inputs and pre-activation gradients, as a
+//                   chunked product with partials added in a fixed order.
+// Nothing is accumulated with atomics: results are reproducible bit for bit.
+// The kernels are dimension-generic (one thread per output element); shapes:
+// two-layer ReLU f and g, single-layer ReLU l_i and h_i, two-layer head with a
+// ReLU hidden layer and a linear output.
+#include <algorithm>
+
+#include "kernels.cuh"
+
+namespace placeto {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRows = 32;          // rows per pass of the row kernels
+
+// ---------------------------------------------------------------- 1. messages
+// FH = relu([H || X] W1 + b1), M = relu(FH W2 + b2) for all rows of one direction.
+__global__ void __launch_bounds__(kThreads)
+grad_messages_kernel(const GradArgs a) {
+    extern __shared__ __align__(16) float smem[];
+    const int dir = blockIdx.y;
+    const DevMlp f = a.f[dir];
+    const int d = a.d, F = a.F, Hf = f.hidden_dim, K = d + F;
+    float *in = smem;                      // [kRows][K]
+    float *hid = in + kRows * K;           // [kRows][Hf]
+    const float *H = a.H[dir];
+    const size_t R = (size_t)a.n * a.B;
+    for (size_t r0 = (size_t)blockIdx.x * kRows; r0 < R; r0 += (size_t)gridDim.x * kRows) {
+        const int rows = (int)min((size_t)kRows, R - r0);
+        for (int i = threadIdx.x; i < rows * K; i += kThreads) {
+            const int r = i / K, k = i - r * K;
+            in[i] = k < d ? H[(r0 + r) * d + k] : a.X[(r0 + r) * F + (k - d)];
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < rows * Hf; i += kThreads) {
+            const int r = i / Hf, j = i - r * Hf;
+            float acc = f.b1[j];
+            for (int k = 0; k < K; ++k) acc = fmaf(in[r * K + k], f.W1[k * Hf + j], acc);
+            acc = fmaxf(acc, 0.f);
+            hid[i] = acc;
+            a.FH[dir][(r0 + r) * Hf + j] = acc;
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < rows * d; i += kThreads) {
+            const int r = i / d, j = i - r * d;
+            float acc = f.b2[j];
+            for (int k = 0; k < Hf; ++k) acc = fmaf(hid[r * Hf + k], f.W2[k * d + j], acc);
+            a.M[dir][(r0 + r) * d + j] = fmaxf(acc, 0.f);
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------- 2. head / pool
+// One block per state (grid-stride). Shared memory: the state's vectors.
+__global__ void __launch_bounds__(kThreads)
+grad_head_kernel(const GradArgs a) {
+    extern __shared__ __align__(16) float smem[];
+    const int d = a.d, F = a.F, m = a.m, n = a.n, B = a.B;
+    const int E = 2 * d + F, Z = 5 * d + F, Hh = a.head.hidden_dim;
+    constexpr int G = kThreads / 32;       // nodes handled per iteration, one warp each
+    float *z = smem;                       // [Z]
+    float *hid = z + Z;                    // [Hh]
+    float *dhid = hid + Hh;                // [Hh]
+    float *dz = dhid + Hh;                 // [Z]
+    float *S = dz + Z;                     // [3][d]
+    float *dS = S + 3 * d;                 // [3][d]
+    float *lg = dS + 3 * d;                // [m] logits, then d/d(logits)
+    float *part = lg + ((m + 3) & ~3);     // [G][3][d] partial sums / [G][d] exchange
+    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+    for (int b = blockIdx.x; b < B; b += gridDim.x) {
+        const int c = a.cur[b];
+        if (c < 0 || c >= n) {             // no such node: the state contributes nothing
+            for (int i = threadIdx.x; i < n * d; i += kThreads) {
+                const size_t off = ((size_t)(i / d) * B + b) * d + (i % d);
+                a.DH[0][off] = 0.f;
+                a.DH[1][off] = 0.f;
+            }
+            for (int k = threadIdx.x; k < Z; k += kThreads) a.Zbuf[(size_t)b * Z + k] = 0.f;
+            for (int k = threadIdx.x; k < Hh; k += kThreads) { a.HID[(size_t)b * Hh + k] = 0.f; a.DHID[(size_t)b * Hh + k] = 0.f; }
+            for (int k = threadIdx.x; k < m; k += kThreads) a.DLOG[(size_t)b * m + k] = 0.f;
+            for (int k = threadIdx.x; k < 3 * d; k += kThreads) { a.Sbuf[(size_t)b * 3 * d + k] = 0.f; a.DPRE_H[(size_t)b * 3 * d + k] = 0.f; }
+            continue;
+        }
+        const uint8_t *rel = a.relation + (size_t)c * n;
+        auto e_of = [&](int u, int k) -> float {
+            return k < d ? a.H[0][((size_t)u * B + b) * d + k]
+                 : k < 2 * d ? a.H[1][((size_t)u * B + b) * d + (k - d)]
+                             : a.X[((size_t)u * B + b) * F + (k - 2 * d)];
+        };
+        // ---- pooled sums S_i = sum_{u in set i} relu(l_i(e_u)); warp g takes nodes g, g + G, ...
+        for (int i = threadIdx.x; i < G * 3 * d; i += kThreads) part[i] = 0.f;
+        __syncthreads();
+        for (int u = g; u < n; u += G) {
+            const int set = rel[u];
+            if (set > 2) continue;
+            const DevMlp &l = a.l[set];
+            for (int j = lane; j < d; j += 32) {
+                float acc = l.b1[j];
+                for (int k = 0; k < E; ++k) acc = fmaf(e_of(u, k), l.W1[k * d + j], acc);
+                part[(g * 3 + set) * d + j] += fmaxf(acc, 0.f);
+            }
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < 3 * d; i += kThreads) {
+            float acc = 0.f;
+            for (int q = 0; q < G; ++q) acc += part[q * 3 * d + i];
+            S[i] = acc;
+            a.Sbuf[(size_t)b * 3 * d + i] = acc;
+        }
+        for (int k = threadIdx.x; k < E; k += kThreads) z[k] = e_of(c, k);
+        __syncthreads();
+        // ---- a_i = relu(h_i(S_i)) into z, hidden layer, logits
+        for (int i = threadIdx.x; i < 3 * d; i += kThreads) {
+            const int set = i / d, j = i - set * d;
+            const DevMlp &h = a.h[set];
+            float acc = h.b1[j];
+            for (int k = 0; k < d; ++k) acc = fmaf(S[set * d + k], h.W1[k * d + j], acc);
+            z[E + i] = fmaxf(acc, 0.f);
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < Hh; j += kThreads) {
+            float acc = a.head.b1[j];
+            for (int k = 0; k < Z; ++k) acc = fmaf(z[k], a.head.W1[(size_t)k * Hh + j], acc);
+            hid[j] = fmaxf(acc, 0.f);
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < m; j += kThreads) {
+            float acc = a.head.b2[j];
+            for (int k = 0; k < Hh; ++k) acc = fmaf(hid[k], a.head.W2[(size_t)k * m + j], acc);
+            lg[j] = acc;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // d/d(logit_k) of A log p[a] + beta H = A (1[k = a] - p_k) - beta p_k (log p_k + H)
+            float mx = lg[0];
+            for (int k = 1; k < m; ++k) mx = fmaxf(mx, lg[k]);
+            float tot = 0.f;
+            for (int k = 0; k < m; ++k) tot += expf(lg[k] - mx);
+            const float lt = logf(tot);
+            float ent = 0.f;
+            for (int k = 0; k < m; ++k) {
+                const float lp = lg[k] - mx - lt;
+                ent -= expf(lp) * lp;
+            }
+            const float A = a.advantages[b];
+            const int act = a.actions[b];
+            for (int k = 0; k < m; ++k) {
+                const float lp = lg[k] - mx - lt, p = expf(lp);
+                lg[k] = A * ((k == act ? 1.f : 0.f) - p) - a.beta * p * (lp + ent);
+            }
+        }
+        __syncthreads();
+        for (int k = threadIdx.x; k < Z; k += kThreads) a.Zbuf[(size_t)b * Z + k] = z[k];
+        for (int j = threadIdx.x; j < m; j += kThreads) a.DLOG[(size_t)b * m + j] = lg[j];
+        for (int k = threadIdx.x; k < Hh; k += kThreads) {
+            float acc = 0.f;
+            for (int j = 0; j < m; ++j) acc = fmaf(lg[j], a.head.W2[(size_t)k * m + j], acc);
+            acc = hid[k] > 0.f ? acc : 0.f;
+            dhid[k] = acc;
+            a.HID[(size_t)b * Hh + k] = hid[k];
+            a.DHID[(size_t)b * Hh + k] = acc;
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < Z; i += kThreads) {
+            float acc = 0.f;
+            for (int k = 0; k < Hh; ++k) acc = fmaf(dhid[k], a.head.W1[(size_t)i * Hh + k], acc);
+            dz[i] = acc;
+        }
+        __syncthreads();
+        // through h_i: dpre_h = dz_a * (a > 0); dS = dpre_h W_h^T
+        for (int i = threadIdx.x; i < 3 * d; i += kThreads) {
+            const float v = z[E + i] > 0.f ? dz[E + i] : 0.f;
+            part[i] = v;
+            a.DPRE_H[(size_t)b * 3 * d + i] = v;
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < 3 * d; i += kThreads) {
+            const int set = i / d, k = i - set * d;
+            const DevMlp &h = a.h[set];
+            float acc = 0.f;
+            for (int j = 0; j < d; ++j) acc = fmaf(part[set * d + j], h.W1[k * d + j], acc);
+            dS[i] = acc;
+        }
+        __syncthreads();
+        // ---- through l_i to every node: dpre_l = dS_set * (pre > 0); de = dpre_l W_l^T
+        float *xch = part;                 // [G][d]
+        for (int u0 = 0; u0 < n; u0 += G) {
+            const int u = u0 + g;
+            const int set = u < n ? rel[u] : 3;
+            if (set <= 2) {
+                const DevMlp &l = a.l[set];
+                for (int j = lane; j < d; j += 32) {
+                    float acc = l.b1[j];
+                    for (int k = 0; k < E; ++k) acc = fmaf(e_of(u, k), l.W1[k * d + j], acc);
+                    const float v = acc > 0.f ? dS[set * d + j] : 0.f;
+                    xch[g * d + j] = v;
+                    a.DPRE_L[set][((size_t)u * B + b) * d + j] = v;
+                }
+            }
+            __syncwarp();
+            if (set <= 2) {
+                const DevMlp &l = a.l[set];
+                for (int k = lane; k < 2 * d; k += 32) {
+                    float acc = 0.f;
+                    for (int j = 0; j < d; ++j) acc = fmaf(xch[g * d + j], l.W1[k * d + j], acc);
+                    float *dst = k < d ? a.DH[0] : a.DH[1];
+                    dst[((size_t)u * B + b) * d + (k < d ? k : k - d)] = acc;
+                }
+            } else if (u < n) {            // the current node: its embedding enters the head directly
+                for (int k = lane; k < 2 * d; k += 32) {
+                    float *dst = k < d ? a.DH[0] : a.DH[1];
+                    dst[((size_t)u * B + b) * d + (k < d ? k : k - d)] = dz[k];
+                }
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ 3. sweeps
+// One block per (state slice, direction): levels in reverse order.
+__global__ void __launch_bounds__(kThreads)
+grad_sweep_kernel(const GradArgs a, int S) {
+    extern __shared__ __align__(16) float smem[];
+    const int dir = blockIdx.y;
+    const DevLevels lv = a.lv[dir];
+    const DevMlp f = a.f[dir], gm = a.g[dir];
+    const int d = a.d, B = a.B, Hf = f.hidden_dim, Hg = gm.hidden_dim;
+    const int b0 = blockIdx.x * S, nb = min(S, B - b0);
+    // consumers of a node's message: children for the top-down pass, parents for the bottom-up one
+    const int *cons_ptr = dir == 0 ? a.child_ptr : a.parent_ptr;
+    const int *cons = dir == 0 ? a.child : a.parent;
+    const int W = max(max(d, Hf), Hg);
+    float *bufA = smem, *bufB = smem + kRows * W, *bufC = bufB + kRows * W;   // [kRows][W] each
+    const float *H = a.H[dir], *M = a.M[dir], *FH = a.FH[dir];
+    for (int level = lv.n_levels - 1; level >= 0; --level) {
+        const int p0 = lv.level_ptr[level], width = lv.level_ptr[level + 1] - p0;
+        const int total = width * nb;
+        for (int r0 = 0; r0 < total; r0 += kRows) {
+            const int rows = min(kRows, total - r0);
+            auto row_of = [&](int r, int &pos, size_t &off) {
+                const int q = (r0 + r) / nb;
+                pos = p0 + q;
+                off = (size_t)lv.order[pos] * B + b0 + (r0 + r - q * nb);
+            };
+            // dpre_f2 = (sum over consumers of ds) * (m > 0)          -> bufA [rows][d]
+            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
+                const int r = i / d, j = i - r * d;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                const int u = lv.order[pos];
+                const int b = (int)(off - (size_t)u * B);
+                float acc = 0.f;
+                for (int e = cons_ptr[u]; e < cons_ptr[u + 1]; ++e)
+                    acc += a.DS[dir][((size_t)cons[e] * B + b) * d + j];
+                acc = M[off * d + j] > 0.f ? acc : 0.f;
+                bufA[r * W + j] = acc;
+                a.DPRE_F2[dir][off * d + j] = acc;
+            }
+            __syncthreads();
+            // dfh = (dpre_f2 W_f2^T) * (fh > 0)                        -> bufB [rows][Hf]
+            for (int i = threadIdx.x; i < rows * Hf; i += kThreads) {
+                const int r = i / Hf, k = i - r * Hf;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                float acc = 0.f;
+                for (int j = 0; j < d; ++j) acc = fmaf(bufA[r * W + j], f.W2[k * d + j], acc);
+                acc = FH[off * Hf + k] > 0.f ? acc : 0.f;
+                bufB[r * W + k] = acc;
+                a.DFH[dir][off * Hf + k] = acc;
+            }
+            __syncthreads();
+            // dh = dH_pool + dfh W_f1[0:d]^T ; dpre_g2 = dh * (h > 0)  -> bufA [rows][d]
+            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
+                const int r = i / d, j = i - r * d;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                float acc = a.DH[dir][off * d + j];
+                for (int k = 0; k < Hf; ++k) acc = fmaf(bufB[r * W + k], f.W1[j * Hf + k], acc);
+                acc = H[off * d + j] > 0.f ? acc : 0.f;
+                a.DPRE_G2[dir][off * d + j] = acc;
+                bufC[r * W + j] = acc;
+            }
+            // s = sum of the neighbours' messages                       -> bufB [rows][d] (after the reads above)
+            __syncthreads();
+            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
+                const int r = i / d, j = i - r * d;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                const int b = (int)(off - (size_t)lv.order[pos] * B);
+                float acc = 0.f;
+                for (int e = lv.nbr_ptr[pos]; e < lv.nbr_ptr[pos + 1]; ++e)
+                    acc += M[((size_t)lv.nbr[e] * B + b) * d + j];
+                bufB[r * W + j] = acc;
+                a.Sg[dir][off * d + j] = acc;
+            }
+            __syncthreads();
+            // t1 = relu(s W_g1 + b) ; dt1 = (dpre_g2 W_g2^T) * (t1 > 0) -> bufA [rows][Hg]
+            for (int i = threadIdx.x; i < rows * Hg; i += kThreads) {
+                const int r = i / Hg, k = i - r * Hg;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                float t1 = gm.b1[k];
+                for (int j = 0; j < d; ++j) t1 = fmaf(bufB[r * W + j], gm.W1[j * Hg + k], t1);
+                t1 = fmaxf(t1, 0.f);
+                float acc = 0.f;
+                for (int j = 0; j < d; ++j) acc = fmaf(bufC[r * W + j], gm.W2[k * d + j], acc);
+                acc = t1 > 0.f ? acc : 0.f;
+                a.T1[dir][off * Hg + k] = t1;
+                a.DT1[dir][off * Hg + k] = acc;
+                bufA[r * W + k] = acc;
+            }
+            __syncthreads();
+            // ds = dt1 W_g1^T                                            -> DS
+            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
+                const int r = i / d, j = i - r * d;
+                int pos; size_t off;
+                row_of(r, pos, off);
+                float acc = 0.f;
+                for (int k = 0; k < Hg; ++k) acc = fmaf(bufA[r * W + k], gm.W1[j * Hg + k], acc);
+                a.DS[dir][off * d + j] = acc;
+            }
+            __syncthreads();
+        }
+        __threadfence_block();
+        __syncthreads();               // the next (lower) level gathers this level's ds
+    }
+}
+
+// ----------------------------------------------------------------- 4. weights
+// partial[chunk][K][J] = sum over the chunk's rows of in[r][k] dp[r][j]; the input
+// row is the concatenation of up to three arrays. Bias: partial_b[chunk][J].
+struct WeightJob {
+    const float *in[3];
+    int width[3], stride[3];     // columns taken from each part, and its row stride
+    const float *dp;
+    int dp_stride;
+    int K, J;
+    size_t R;
+    float *partial;       // [chunks][(K + 1) * J], row K holds the bias sums
+    float *dW, *db;
+    int chunks;
+};
+
+__global__ void __launch_bounds__(kThreads)
+grad_weight_partial_kernel(const WeightJob w) {
+    extern __shared__ __align__(16) float smem[];
+    const int K = w.K, J = w.J;
+    float *in = smem;                  // [kRows][K + 1] (last column = 1 for the bias)
+    float *dp = in + kRows * (K + 1);  // [kRows][J]
+    const int chunk = blockIdx.x;
+    const size_t per = (w.R + w.chunks - 1) / w.chunks;
+    const size_t r_begin = (size_t)chunk * per, r_end = min(w.R, r_begin + per);
+    const int tile0 = blockIdx.y * 1024;                 // output elements [tile0, tile0 + 1024)
+    const int n_out = (K + 1) * J;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};                 // elements tile0 + threadIdx.x + 256 q
+    for (size_t r0 = r_begin; r0 < r_end; r0 += kRows) {
+        const int rows = (int)min((size_t)kRows, r_end - r0);
+        for (int i = threadIdx.x; i < rows * (K + 1); i += kThreads) {
+            const int r = i / (K + 1), k = i - r * (K + 1);
+            float v = 1.f;
+            if (k < K) {
+                int kk = k, part = 0;
+                while (kk >= w.width[part]) { kk -= w.width[part]; ++part; }
+                v = w.in[part][(r0 + r) * w.stride[part] + kk];
+            }
+            in[i] = v;
+        }
+        for (int i = threadIdx.x; i < rows * J; i += kThreads) {
+            const int r = i / J, j = i - r * J;
+            dp[i] = w.dp[(r0 + r) * w.dp_stride + j];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int o = tile0 + threadIdx.x + kThreads * q;
+            if (o < n_out) {
+                const int k = o / J, j = o - k * J;
+                float s = acc[q];
+                for (int r = 0; r < rows; ++r) s = fmaf(in[r * (K + 1) + k], dp[r * J + j], s);
+                acc[q] = s;
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int o = tile0 + threadIdx.x + kThreads * q;
+        if (o < n_out) w.partial[(size_t)chunk * n_out + o] = acc[q];
+    }
+}
+
+__global__ void grad_weight_reduce_kernel(const WeightJob w) {
+    const int n_out = (w.K + 1) * w.J;
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= n_out) return;
+    float acc = 0.f;
+    for (int c = 0; c < w.chunks; ++c) acc += w.partial[(size_t)c * n_out + o];   // ascending: fixed order
+    if (o < w.K * w.J) w.dW[o] = acc;
+    else w.db[o - w.K * w.J] = acc;
+}
+
+cudaError_t weight_grad(WeightJob w, cudaStream_t stream) {
+    const size_t smem = ((size_t)kRows * (w.K + 1) + (size_t)kRows * w.J) * sizeof(float);
+    cudaError_t err = cudaFuncSetAttribute(grad_weight_partial_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    const int n_out = (w.K + 1) * w.J;
+    grad_weight_partial_kernel<<<dim3(w.chunks, (n_out + 1023) / 1024), kThreads, smem, stream>>>(w);
+    count_launch();
+    grad_weight_reduce_kernel<<<(n_out + 255) / 256, 256, 0, stream>>>(w);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool policy_gradient_applicable(const GradArgs &a) {
+    auto relu2 = [](const DevMlp &m) { return m.n_layers == 2 && m.act == 0 && m.final_act == 1; };
+    auto relu1 = [](const DevMlp &m) { return m.n_layers == 1 && m.act == 0 && m.final_act == 1; };
+    for (int dir = 0; dir < 2; ++dir)
+        if (!relu2(a.f[dir]) || !relu2(a.g[dir])) return false;
+    for (int i = 0; i < 3; ++i)
+        if (!relu1(a.l[i]) || !relu1(a.h[i])) return false;
+    return a.head.n_layers == 2 && a.head.act == 0 && a.head.final_act == 0;
+}
+
+// floats of workspace (every array padded to a multiple of 4 floats by the carve below)
+size_t policy_gradient_workspace_floats(int n, int B, int d, int F, int m, int Hf, int Hg, int Hh) {
+    const size_t R = (size_t)n * B, Z = 5 * (size_t)d + F, E = 2 * (size_t)d + F;
+    const size_t per_dir = R * ((size_t)Hf * 2 + (size_t)Hg * 2 + (size_t)d * 6);
+    size_t total = 2 * per_dir + 3 * R * d;
+    total += (size_t)B * (Z + 2 * (size_t)Hh + m + 6 * (size_t)d);
+    size_t widest = std::max((Z + 1) * (size_t)Hh, ((size_t)Hh + 1) * m);
+    widest = std::max({widest, (E + 1) * (size_t)d, ((size_t)d + F + 1) * Hf, ((size_t)Hf + 1) * d,
+                       ((size_t)d + 1) * Hg, ((size_t)Hg + 1) * d});
+    return total + (size_t)kGradChunks * widest + 256;
+}
+
+cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, cudaStream_t stream) {
+    const int n = a.n, B = a.B, d = a.d, F = a.F, m = a.m;
+    const size_t R = (size_t)n * B;
+    const int Z = 5 * d + F, Hh = a.head.hidden_dim;
+    float *p = ws;
+    auto take = [&](size_t floats) { float *q = p; p += (floats + 3) & ~size_t(3); return q; };
+    for (int dir = 0; dir < 2; ++dir) {
+        const int Hf = a.f[dir].hidden_dim, Hg = a.g[dir].hidden_dim;
+        a.FH[dir] = take(R * Hf); a.DFH[dir] = take(R * Hf);
+        a.T1[dir] = take(R * Hg); a.DT1[dir] = take(R * Hg);
+        a.M[dir] = take(R * d); a.DS[dir] = take(R * d);
+        a.DPRE_F2[dir] = take(R * d); a.DPRE_G2[dir] = take(R * d);
+        a.Sg[dir] = take(R * d); a.DH[dir] = take(R * d);
+    }
+    for (int i = 0; i < 3; ++i) a.DPRE_L[i] = take(R * d);
+    a.Zbuf = take((size_t)B * Z); a.HID = take((size_t)B * Hh); a.DHID = take((size_t)B * Hh);
+    a.DLOG = take((size_t)B * m); a.Sbuf = take((size_t)B * 3 * d); a.DPRE_H = take((size_t)B * 3 * d);
+    float *partial = p;
+
+    cudaError_t err = cudaMemsetAsync(a.DPRE_L[0], 0, 3 * ((R * d + 3) & ~size_t(3)) * sizeof(float), stream);
+    if (err != cudaSuccess) return err;
+    // 1. messages
+    {
+        const int Hf = std::max(a.f[0].hidden_dim, a.f[1].hidden_dim);
+        const size_t smem = (size_t)kRows * (d + F + Hf) * sizeof(float);
+        err = cudaFuncSetAttribute(grad_messages_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        const int blocks = (int)std::min<size_t>((R + kRows - 1) / kRows, 4 * (size_t)di.sm_count);
+        grad_messages_kernel<<<dim3(blocks, 2), kThreads, smem, stream>>>(a);
+        count_launch();
+    }
+    // 2. head and pooling
+    {
+        const size_t floats = 2 * (size_t)Z + 2 * (size_t)Hh + 6 * (size_t)d + ((m + 3) & ~3) +
+                              (size_t)(kThreads / 32) * 3 * d;
+        const size_t smem = floats * sizeof(float);
+        err = cudaFuncSetAttribute(grad_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        grad_head_kernel<<<std::min(B, 8 * di.sm_count), kThreads, smem, stream>>>(a);
+        count_launch();
+    }
+    // 3. reverse sweeps
+    {
+        const int slices = std::max(1, std::min(B, di.sm_count / 2));
+        const int S = (B + slices - 1) / slices;
+        int W = d;
+        for (int dir = 0; dir < 2; ++dir) W = std::max({W, a.f[dir].hidden_dim, a.g[dir].hidden_dim});
+        const size_t smem = 3 * (size_t)kRows * W * sizeof(float);
+        err = cudaFuncSetAttribute(grad_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        grad_sweep_kernel<<<dim3((B + S - 1) / S, 2), kThreads, smem, stream>>>(a, S);
+        count_launch();
+    }
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    // 4. weight gradients: dW = in^T dpre, db = sum dpre
+    auto job = [&](const float *in0, int w0, const float *in1, int w1, const float *in2, int w2,
+                   const float *dp, int J, size_t rows, float *dW, float *db) {
+        WeightJob w;
+        w.in[0] = in0; w.in[1] = in1; w.in[2] = in2;
+        w.width[0] = w0; w.width[1] = w1; w.width[2] = w2;
+        w.stride[0] = w0; w.stride[1] = w1; w.stride[2] = w2;
+        w.dp = dp; w.dp_stride = J; w.K = w0 + w1 + w2; w.J = J; w.R = rows;
+        w.partial = partial; w.dW = dW; w.db = db;
+        w.chunks = (int)std::max<size_t>(1, std::min<size_t>(kGradChunks, (rows + kRows - 1) / kRows));
+        return weight_grad(w, stream);
+    };
+    for (int dir = 0; dir < 2 && err == cudaSuccess; ++dir) {
+        const int Hf = a.f[dir].hidden_dim, Hg = a.g[dir].hidden_dim;
+        err = job(a.H[dir], d, a.X, F, nullptr, 0, a.DFH[dir], Hf, R, a.gf[dir].W1, a.gf[dir].b1);
+        if (err == cudaSuccess) err = job(a.FH[dir], Hf, nullptr, 0, nullptr, 0, a.DPRE_F2[dir], d, R, a.gf[dir].W2, a.gf[dir].b2);
+        if (err == cudaSuccess) err = job(a.Sg[dir], d, nullptr, 0, nullptr, 0, a.DT1[dir], Hg, R, a.gg[dir].W1, a.gg[dir].b1);
+        if (err == cudaSuccess) err = job(a.T1[dir], Hg, nullptr, 0, nullptr, 0, a.DPRE_G2[dir], d, R, a.gg[dir].W2, a.gg[dir].b2);
+    }
+    for (int i = 0; i < 3 && err == cudaSuccess; ++i) {
+        err = job(a.H[0], d, a.H[1], d, a.X, F, a.DPRE_L[i], d, R, a.gl[i].W1, a.gl[i].b1);
+        // h_i: rows are states; the inputs and gradients of set i sit at column offset i * d of [B][3][d]
+        if (err == cudaSuccess) {
+            WeightJob w;
+            w.in[0] = a.Sbuf + i * d; w.in[1] = w.in[2] = nullptr;
+            w.width[0] = d; w.width[1] = w.width[2] = 0;
+            w.stride[0] = 3 * d; w.stride[1] = w.stride[2] = 0;
+            w.dp = a.DPRE_H + i * d; w.dp_stride = 3 * d; w.K = d; w.J = d; w.R = B;
+            w.partial = partial; w.dW = a.gh[i].W1; w.db = a.gh[i].b1;
+            w.chunks = 1;
+            err = weight_grad(w, stream);
+        }
+    }
+    if (err == cudaSuccess) err = job(a.Zbuf, Z, nullptr, 0, nullptr, 0, a.DHID, Hh, B, a.ghead.W1, a.ghead.b1);
+    if (err == cudaSuccess) err = job(a.HID, Hh, nullptr, 0, nullptr, 0, a.DLOG, m, B, a.ghead.W2, a.ghead.b2);
+    return err;
+}
+
+}  // namespace placeto

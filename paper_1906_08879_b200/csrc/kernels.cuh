@@ -88,6 +88,24 @@ struct SimArgs {
     char *workspace;
 };
 
+// Policy gradient (gradient.cu): inputs, per-row intermediates in the workspace, outputs.
+constexpr int kGradChunks = 64;    // row chunks whose partial weight gradients are added in order
+struct GradOut { float *W1, *b1, *W2, *b2; };
+struct GradArgs {
+    int n, B, d, F, m;
+    const uint8_t *relation;
+    DevLevels lv[2];
+    const int *child_ptr, *child, *parent_ptr, *parent;   // by node id
+    DevMlp f[2], g[2], l[3], h[3], head;
+    const float *X, *H[2];
+    const int *cur, *actions;
+    const float *advantages;
+    float beta;
+    float *FH[2], *DFH[2], *T1[2], *DT1[2], *M[2], *DS[2], *DPRE_F2[2], *DPRE_G2[2], *Sg[2], *DH[2];
+    float *DPRE_L[3], *Zbuf, *HID, *DHID, *DLOG, *Sbuf, *DPRE_H;
+    GradOut gf[2], gg[2], gl[3], gh[3], ghead;
+};
+
 struct DeviceInfo {
     int sm_count;
     int max_smem_optin;   // bytes per block
@@ -138,6 +156,11 @@ cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream
 // simulator.cu: event-based run time of P placements, one thread each
 size_t sim_workspace_bytes(int n, int n_edges, int m, int P);
 cudaError_t launch_simulator(const SimArgs &a, cudaStream_t stream);
+
+// gradient.cu: gradient of the policy objective with respect to all weights
+bool policy_gradient_applicable(const GradArgs &a);
+size_t policy_gradient_workspace_floats(int n, int B, int d, int F, int m, int Hf, int Hg, int Hh);
+cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, cudaStream_t stream);
 
 // embed_generic.cu: dimension-generic message passing. schedule is one of
 // PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.

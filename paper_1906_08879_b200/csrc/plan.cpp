@@ -125,6 +125,12 @@ placeto_status build_plan(int32_t n, int64_t n_edges, const int32_t *src, const 
             plan.child_ptr[v + 1] = static_cast<int32_t>(plan.child.size());
             plan.n_parents[v] = static_cast<int32_t>(par[v].size());
         }
+        plan.parent_ptr.assign(n + 1, 0);
+        plan.parent.clear();
+        for (int32_t v = 0; v < n; ++v) {
+            plan.parent.insert(plan.parent.end(), par[v].begin(), par[v].end());
+            plan.parent_ptr[v + 1] = static_cast<int32_t>(plan.parent.size());
+        }
         plan.max_level_width = 0;
         for (int dir = 0; dir < 2; ++dir)
             for (int32_t l = 0; l < plan.dir[dir].n_levels; ++l)

@@ -33,6 +33,7 @@ struct HostPlan {
     std::vector<uint8_t> relation;   // [n * n], see placeto_graph_host_view
     // by node id, for the runtime simulator: children (ascending) and number of parents
     std::vector<int32_t> child_ptr, child, n_parents;
+    std::vector<int32_t> parent_ptr, parent;   // by node id, ascending (the policy gradient's gathers)
 };
 
 // Validates the edge list and fills `plan`. Returns PLACETO_OK,
