@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--rounds", type=int, default=0,
                     help="K > 0: the message-passing launch timed alone (roofline) is placeto_embed_rounds "
                          "with K synchronous rounds instead of the progressive sweep")
+    ap.add_argument("--gradient", action="store_true",
+                    help="instead of the policy path, time placeto_policy_gradient (the backward of one batch, "
+                         "embeddings given) on the workload; own JSON line")
     ap.add_argument("--simulate", type=int, default=0,
                     help="P > 0: instead of the policy path, time placeto_simulate_runtime on P random "
                          "placements of the workload's graph (its own metric: simulated placements/s)")
@@ -484,8 +487,53 @@ def run_simulator(args):
     return 0
 
 
+def run_gradient(args):
+    """Extra mode: the policy gradient of one batch (forward intermediates X, H given)."""
+    import torch
+    import paper_1906_08879_b200 as placeto
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    cfg = make_workload(args.workload)
+    n, B, m = cfg["n"], cfg["B"], cfg["m"]
+    g = placeto.Graph(n, cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    dev_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    cur = dev_t(cfg["cur"])
+    X = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]), cur,
+                                       dev_t(cfg["placed"]), m)
+    Hd, Hu = placeto.placeto_embed_forward(g, w, X)
+    rng = np.random.Generator(np.random.PCG64(7))
+    actions = dev_t(rng.integers(0, m, B).astype(np.int32))
+    adv = dev_t(rng.normal(size=B).astype(np.float32))
+    grads = placeto.binding.zero_gradients(cfg["weights"])
+    ws = placeto.workspace(g, w, B, placeto.CALL_GRADIENT)
+    stream = torch.cuda.current_stream()
+    run = lambda: placeto.placeto_policy_gradient(g, w, X, Hd, Hu, cur, actions, adv, 0.01, grads, ws, stream)
+    for _ in range(max(args.warmup, 3)):
+        run()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record(stream)
+    for _ in range(args.steps):
+        run()
+    e.record(stream)
+    torch.cuda.synchronize()
+    ms = s.elapsed_time(e) / args.steps
+    d, F = cfg["d"], cfg["F"]
+    flop = 3.0 * (flops_embed(cfg) + flops_pool(cfg))      # recompute + two products per forward product
+    print(json.dumps({"metric": "states differentiated/sec (policy gradient, embeddings given)",
+                      "value": B / (ms * 1e-3), "unit": "states/s", "n_gpus": 1, "steps": args.steps,
+                      "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+                      "gpu_launches": placeto.placeto_last_launch_count(),
+                      "config": {"workload": cfg["name"] + "-gradient", "n_nodes": n, "states": B, "d": d, "F": F,
+                                 "workspace_bytes": int(ws.numel())},
+                      "approx_tflops": flop / (ms * 1e-3) / 1e12}))
+    return 0
+
+
 def main():
     args = parse_args()
+    if args.gradient and args.impl != "reference":
+        return run_gradient(args)
     if args.simulate > 0 and args.impl != "reference":
         return run_simulator(args)
     if args.impl == "reference":

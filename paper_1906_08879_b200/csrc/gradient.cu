@@ -251,6 +251,20 @@ grad_sweep_kernel(const GradArgs a, int S) {
     const int *cons = dir == 0 ? a.child : a.parent;
     const int W = max(max(d, Hf), Hg);
     float *bufA = smem, *bufB = smem + kRows * W, *bufC = bufB + kRows * W;   // [kRows][W] each
+    // the direction's matrices in shared memory, rows padded by one float so that
+    // both the row-wise and the column-wise reads below are free of bank conflicts
+    const int sf = Hf + 1, sd = d + 1, sg = Hg + 1;
+    float *wf1 = bufC + kRows * W;         // [d][Hf]: the h rows of f's first layer
+    float *wf2 = wf1 + d * sf;             // [Hf][d]
+    float *wg1 = wf2 + Hf * sd;            // [d][Hg]
+    float *wg2 = wg1 + d * sg;             // [Hg][d]
+    float *bg1 = wg2 + Hg * sd;            // [Hg]
+    for (int i = threadIdx.x; i < d * Hf; i += kThreads) wf1[(i / Hf) * sf + i % Hf] = f.W1[i];
+    for (int i = threadIdx.x; i < Hf * d; i += kThreads) wf2[(i / d) * sd + i % d] = f.W2[i];
+    for (int i = threadIdx.x; i < d * Hg; i += kThreads) wg1[(i / Hg) * sg + i % Hg] = gm.W1[i];
+    for (int i = threadIdx.x; i < Hg * d; i += kThreads) wg2[(i / d) * sd + i % d] = gm.W2[i];
+    for (int i = threadIdx.x; i < Hg; i += kThreads) bg1[i] = gm.b1[i];
+    __syncthreads();
     const float *H = a.H[dir], *M = a.M[dir], *FH = a.FH[dir];
     for (int level = lv.n_levels - 1; level >= 0; --level) {
         const int p0 = lv.level_ptr[level], width = lv.level_ptr[level + 1] - p0;
@@ -283,7 +297,7 @@ grad_sweep_kernel(const GradArgs a, int S) {
                 int pos; size_t off;
                 row_of(r, pos, off);
                 float acc = 0.f;
-                for (int j = 0; j < d; ++j) acc = fmaf(bufA[r * W + j], f.W2[k * d + j], acc);
+                for (int j = 0; j < d; ++j) acc = fmaf(bufA[r * W + j], wf2[k * sd + j], acc);
                 acc = FH[off * Hf + k] > 0.f ? acc : 0.f;
                 bufB[r * W + k] = acc;
                 a.DFH[dir][off * Hf + k] = acc;
@@ -295,7 +309,7 @@ grad_sweep_kernel(const GradArgs a, int S) {
                 int pos; size_t off;
                 row_of(r, pos, off);
                 float acc = a.DH[dir][off * d + j];
-                for (int k = 0; k < Hf; ++k) acc = fmaf(bufB[r * W + k], f.W1[j * Hf + k], acc);
+                for (int k = 0; k < Hf; ++k) acc = fmaf(bufB[r * W + k], wf1[j * sf + k], acc);
                 acc = H[off * d + j] > 0.f ? acc : 0.f;
                 a.DPRE_G2[dir][off * d + j] = acc;
                 bufC[r * W + j] = acc;
@@ -319,11 +333,11 @@ grad_sweep_kernel(const GradArgs a, int S) {
                 const int r = i / Hg, k = i - r * Hg;
                 int pos; size_t off;
                 row_of(r, pos, off);
-                float t1 = gm.b1[k];
-                for (int j = 0; j < d; ++j) t1 = fmaf(bufB[r * W + j], gm.W1[j * Hg + k], t1);
+                float t1 = bg1[k];
+                for (int j = 0; j < d; ++j) t1 = fmaf(bufB[r * W + j], wg1[j * sg + k], t1);
                 t1 = fmaxf(t1, 0.f);
                 float acc = 0.f;
-                for (int j = 0; j < d; ++j) acc = fmaf(bufC[r * W + j], gm.W2[k * d + j], acc);
+                for (int j = 0; j < d; ++j) acc = fmaf(bufC[r * W + j], wg2[k * sd + j], acc);
                 acc = t1 > 0.f ? acc : 0.f;
                 a.T1[dir][off * Hg + k] = t1;
                 a.DT1[dir][off * Hg + k] = acc;
@@ -336,7 +350,7 @@ grad_sweep_kernel(const GradArgs a, int S) {
                 int pos; size_t off;
                 row_of(r, pos, off);
                 float acc = 0.f;
-                for (int k = 0; k < Hg; ++k) acc = fmaf(bufA[r * W + k], gm.W1[j * Hg + k], acc);
+                for (int k = 0; k < Hg; ++k) acc = fmaf(bufA[r * W + k], wg1[j * sg + k], acc);
                 a.DS[dir][off * d + j] = acc;
             }
             __syncthreads();
@@ -503,7 +517,13 @@ cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, 
         const int S = (B + slices - 1) / slices;
         int W = d;
         for (int dir = 0; dir < 2; ++dir) W = std::max({W, a.f[dir].hidden_dim, a.g[dir].hidden_dim});
-        const size_t smem = 3 * (size_t)kRows * W * sizeof(float);
+        size_t wfloats = 0;
+        for (int dir = 0; dir < 2; ++dir) {
+            const size_t Hf = a.f[dir].hidden_dim, Hg = a.g[dir].hidden_dim;
+            wfloats = std::max(wfloats, d * (Hf + 1) + Hf * ((size_t)d + 1) + d * (Hg + 1) + Hg * ((size_t)d + 1) + Hg);
+        }
+        const size_t smem = (3 * (size_t)kRows * W + wfloats) * sizeof(float);
+        if (smem > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
         err = cudaFuncSetAttribute(grad_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         grad_sweep_kernel<<<dim3((B + S - 1) / S, 2), kThreads, smem, stream>>>(a, S);

@@ -89,7 +89,7 @@ struct SimArgs {
 };
 
 // Policy gradient (gradient.cu): inputs, per-row intermediates in the workspace, outputs.
-constexpr int kGradChunks = 64;    // row chunks whose partial weight gradients are added in order
+constexpr int kGradChunks = 256;   // row chunks whose partial weight gradients are added in order
 struct GradOut { float *W1, *b1, *W2, *b2; };
 struct GradArgs {
     int n, B, d, F, m;
