@@ -84,7 +84,16 @@ grad_head_kernel(const GradArgs a) {
     float *dS = S + 3 * d;                 // [3][d]
     float *lg = dS + 3 * d;                // [m] logits, then d/d(logits)
     float *part = lg + ((m + 3) & ~3);     // [G][3][d] partial sums / [G][d] exchange
+    float *erow = part + G * 3 * d;        // [G][E]: the embedding row a warp is working on
+    float *wl = erow + G * ((E + 3) & ~3); // [3][E * d + d]: the three l_i (weights, then bias)
     const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const int lsz = E * d + d;
+    for (int i = 0; i < 3; ++i) {
+        for (int t = threadIdx.x; t < E * d; t += kThreads) wl[i * lsz + t] = a.l[i].W1[t];
+        for (int t = threadIdx.x; t < d; t += kThreads) wl[i * lsz + E * d + t] = a.l[i].b1[t];
+    }
+    float *my_e = erow + g * ((E + 3) & ~3);
+    __syncthreads();
     for (int b = blockIdx.x; b < B; b += gridDim.x) {
         const int c = a.cur[b];
         if (c < 0 || c >= n) {             // no such node: the state contributes nothing
@@ -111,10 +120,13 @@ grad_head_kernel(const GradArgs a) {
         for (int u = g; u < n; u += G) {
             const int set = rel[u];
             if (set > 2) continue;
-            const DevMlp &l = a.l[set];
+            const float *W = wl + set * lsz;
+            __syncwarp();
+            for (int k = lane; k < E; k += 32) my_e[k] = e_of(u, k);
+            __syncwarp();
             for (int j = lane; j < d; j += 32) {
-                float acc = l.b1[j];
-                for (int k = 0; k < E; ++k) acc = fmaf(e_of(u, k), l.W1[k * d + j], acc);
+                float acc = W[E * d + j];
+                for (int k = 0; k < E; ++k) acc = fmaf(my_e[k], W[k * d + j], acc);
                 part[(g * 3 + set) * d + j] += fmaxf(acc, 0.f);
             }
         }
@@ -138,6 +150,7 @@ grad_head_kernel(const GradArgs a) {
         __syncthreads();
         for (int j = threadIdx.x; j < Hh; j += kThreads) {
             float acc = a.head.b1[j];
+#pragma unroll 8
             for (int k = 0; k < Z; ++k) acc = fmaf(z[k], a.head.W1[(size_t)k * Hh + j], acc);
             hid[j] = fmaxf(acc, 0.f);
         }
@@ -179,10 +192,12 @@ grad_head_kernel(const GradArgs a) {
             a.DHID[(size_t)b * Hh + k] = acc;
         }
         __syncthreads();
-        for (int i = threadIdx.x; i < Z; i += kThreads) {
+        for (int i = g; i < Z; i += G) {       // a warp per input: its weight row is contiguous
             float acc = 0.f;
-            for (int k = 0; k < Hh; ++k) acc = fmaf(dhid[k], a.head.W1[(size_t)i * Hh + k], acc);
-            dz[i] = acc;
+            for (int k = lane; k < Hh; k += 32) acc = fmaf(dhid[k], a.head.W1[(size_t)i * Hh + k], acc);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) dz[i] = acc;
         }
         __syncthreads();
         // through h_i: dpre_h = dz_a * (a > 0); dS = dpre_h W_h^T
@@ -206,10 +221,12 @@ grad_head_kernel(const GradArgs a) {
             const int u = u0 + g;
             const int set = u < n ? rel[u] : 3;
             if (set <= 2) {
-                const DevMlp &l = a.l[set];
+                const float *W = wl + set * lsz;
+                for (int k = lane; k < E; k += 32) my_e[k] = e_of(u, k);
+                __syncwarp();
                 for (int j = lane; j < d; j += 32) {
-                    float acc = l.b1[j];
-                    for (int k = 0; k < E; ++k) acc = fmaf(e_of(u, k), l.W1[k * d + j], acc);
+                    float acc = W[E * d + j];
+                    for (int k = 0; k < E; ++k) acc = fmaf(my_e[k], W[k * d + j], acc);
                     const float v = acc > 0.f ? dS[set * d + j] : 0.f;
                     xch[g * d + j] = v;
                     a.DPRE_L[set][((size_t)u * B + b) * d + j] = v;
@@ -217,10 +234,13 @@ grad_head_kernel(const GradArgs a) {
             }
             __syncwarp();
             if (set <= 2) {
-                const DevMlp &l = a.l[set];
+                const float *W = wl + set * lsz;
                 for (int k = lane; k < 2 * d; k += 32) {
                     float acc = 0.f;
-                    for (int j = 0; j < d; ++j) acc = fmaf(xch[g * d + j], l.W1[k * d + j], acc);
+                    for (int j = 0; j < d; ++j) {
+                        const int jj = (j + lane) % d;     // rotated per lane: no shared-memory bank conflicts
+                        acc = fmaf(xch[g * d + jj], W[k * d + jj], acc);
+                    }
                     float *dst = k < d ? a.DH[0] : a.DH[1];
                     dst[((size_t)u * B + b) * d + (k < d ? k : k - d)] = acc;
                 }
@@ -423,14 +443,26 @@ grad_weight_partial_kernel(const WeightJob w) {
     }
 }
 
-__global__ void grad_weight_reduce_kernel(const WeightJob w) {
+// Adds the chunk partials: a block owns 32 outputs; eight thread groups each add
+// every eighth chunk (ascending), then the eight sums are added in group order.
+__global__ void __launch_bounds__(256)
+grad_weight_reduce_kernel(const WeightJob w) {
+    __shared__ float sums[8][32];
     const int n_out = (w.K + 1) * w.J;
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= n_out) return;
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + lane;
     float acc = 0.f;
-    for (int c = 0; c < w.chunks; ++c) acc += w.partial[(size_t)c * n_out + o];   // ascending: fixed order
-    if (o < w.K * w.J) w.dW[o] = acc;
-    else w.db[o - w.K * w.J] = acc;
+    if (o < n_out)
+        for (int c = grp; c < w.chunks; c += 8) acc += w.partial[(size_t)c * n_out + o];
+    sums[grp][lane] = acc;
+    __syncthreads();
+    if (grp == 0 && o < n_out) {
+        float total = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) total += sums[q][lane];
+        if (o < w.K * w.J) w.dW[o] = total;
+        else w.db[o - w.K * w.J] = total;
+    }
 }
 
 cudaError_t weight_grad(WeightJob w, cudaStream_t stream) {
@@ -441,7 +473,7 @@ cudaError_t weight_grad(WeightJob w, cudaStream_t stream) {
     const int n_out = (w.K + 1) * w.J;
     grad_weight_partial_kernel<<<dim3(w.chunks, (n_out + 1023) / 1024), kThreads, smem, stream>>>(w);
     count_launch();
-    grad_weight_reduce_kernel<<<(n_out + 255) / 256, 256, 0, stream>>>(w);
+    grad_weight_reduce_kernel<<<(n_out + 31) / 32, 256, 0, stream>>>(w);
     count_launch();
     return cudaGetLastError();
 }
@@ -503,8 +535,10 @@ cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, 
     }
     // 2. head and pooling
     {
+        const size_t E = 2 * (size_t)d + F;
         const size_t floats = 2 * (size_t)Z + 2 * (size_t)Hh + 6 * (size_t)d + ((m + 3) & ~3) +
-                              (size_t)(kThreads / 32) * 3 * d;
+                              (size_t)(kThreads / 32) * 3 * d + (size_t)(kThreads / 32) * ((E + 3) & ~size_t(3)) +
+                              3 * (E * d + d);
         const size_t smem = floats * sizeof(float);
         err = cudaFuncSetAttribute(grad_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
