@@ -395,9 +395,19 @@ struct WeightJob {
     int chunks;
 };
 
+constexpr int kMaxJobs = 16;
+struct WeightJobs {
+    WeightJob job[kMaxJobs];
+    int count;
+};
+
+// All layers in one launch: blockIdx.z picks the job, blocks beyond a job's
+// chunks or output tiles leave at once.
 __global__ void __launch_bounds__(kThreads)
-grad_weight_partial_kernel(const WeightJob w) {
+grad_weight_partial_kernel(const WeightJobs jobs) {
     extern __shared__ __align__(16) float smem[];
+    const WeightJob &w = jobs.job[blockIdx.z];
+    if ((int)blockIdx.x >= w.chunks || (int)blockIdx.y * 1024 >= (w.K + 1) * w.J) return;
     const int K = w.K, J = w.J;
     float *in = smem;                  // [kRows][K + 1] (last column = 1 for the bias)
     float *dp = in + kRows * (K + 1);  // [kRows][J]
@@ -446,9 +456,11 @@ grad_weight_partial_kernel(const WeightJob w) {
 // Adds the chunk partials: a block owns 32 outputs; eight thread groups each add
 // every eighth chunk (ascending), then the eight sums are added in group order.
 __global__ void __launch_bounds__(256)
-grad_weight_reduce_kernel(const WeightJob w) {
+grad_weight_reduce_kernel(const WeightJobs jobs) {
     __shared__ float sums[8][32];
+    const WeightJob &w = jobs.job[blockIdx.y];
     const int n_out = (w.K + 1) * w.J;
+    if ((int)blockIdx.x * 32 >= n_out) return;
     const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
     const int o = blockIdx.x * 32 + lane;
     float acc = 0.f;
@@ -465,15 +477,22 @@ grad_weight_reduce_kernel(const WeightJob w) {
     }
 }
 
-cudaError_t weight_grad(WeightJob w, cudaStream_t stream) {
-    const size_t smem = ((size_t)kRows * (w.K + 1) + (size_t)kRows * w.J) * sizeof(float);
+cudaError_t weight_grads(const WeightJobs &jobs, cudaStream_t stream) {
+    if (jobs.count == 0) return cudaSuccess;
+    size_t smem = 0;
+    int max_chunks = 1, max_out = 1;
+    for (int i = 0; i < jobs.count; ++i) {
+        const WeightJob &w = jobs.job[i];
+        smem = std::max(smem, ((size_t)kRows * (w.K + 1) + (size_t)kRows * w.J) * sizeof(float));
+        max_chunks = std::max(max_chunks, w.chunks);
+        max_out = std::max(max_out, (w.K + 1) * w.J);
+    }
     cudaError_t err = cudaFuncSetAttribute(grad_weight_partial_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    const int n_out = (w.K + 1) * w.J;
-    grad_weight_partial_kernel<<<dim3(w.chunks, (n_out + 1023) / 1024), kThreads, smem, stream>>>(w);
+    grad_weight_partial_kernel<<<dim3(max_chunks, (max_out + 1023) / 1024, jobs.count), kThreads, smem, stream>>>(jobs);
     count_launch();
-    grad_weight_reduce_kernel<<<(n_out + 31) / 32, 256, 0, stream>>>(w);
+    grad_weight_reduce_kernel<<<dim3((max_out + 31) / 32, jobs.count), 256, 0, stream>>>(jobs);
     count_launch();
     return cudaGetLastError();
 }
@@ -496,9 +515,9 @@ size_t policy_gradient_workspace_floats(int n, int B, int d, int F, int m, int H
     const size_t per_dir = R * ((size_t)Hf * 2 + (size_t)Hg * 2 + (size_t)d * 6);
     size_t total = 2 * per_dir + 3 * R * d;
     total += (size_t)B * (Z + 2 * (size_t)Hh + m + 6 * (size_t)d);
-    size_t widest = std::max((Z + 1) * (size_t)Hh, ((size_t)Hh + 1) * m);
-    widest = std::max({widest, (E + 1) * (size_t)d, ((size_t)d + F + 1) * Hf, ((size_t)Hf + 1) * d,
-                       ((size_t)d + 1) * Hg, ((size_t)Hg + 1) * d});
+    // chunk partials of all sixteen layer products side by side
+    const size_t widest = 2 * (((size_t)d + F + 1) * Hf + ((size_t)Hf + 1) * d + ((size_t)d + 1) * Hg + ((size_t)Hg + 1) * d) +
+                          3 * ((E + 1) * (size_t)d + ((size_t)d + 1) * d) + (Z + 1) * (size_t)Hh + ((size_t)Hh + 1) * m;
     return total + (size_t)kGradChunks * widest + 256;
 }
 
@@ -565,42 +584,41 @@ cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, 
     }
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    // 4. weight gradients: dW = in^T dpre, db = sum dpre
-    auto job = [&](const float *in0, int w0, const float *in1, int w1, const float *in2, int w2,
-                   const float *dp, int J, size_t rows, float *dW, float *db) {
-        WeightJob w;
+    // 4. weight gradients: dW = in^T dpre, db = sum dpre, every layer in one launch
+    // two launches: the layers summed over all (node, state) rows, and those summed over
+    // states only (the head's wide matrices would otherwise set every block's shared memory)
+    WeightJobs by_row, by_state;
+    by_row.count = by_state.count = 0;
+    auto job = [&](const float *in0, int w0, int s0, const float *in1, int w1, const float *in2, int w2,
+                   const float *dp, int dp_stride, int J, size_t rows, float *dW, float *db) {
+        WeightJobs &list = rows == R ? by_row : by_state;
+        WeightJob &w = list.job[list.count++];
         w.in[0] = in0; w.in[1] = in1; w.in[2] = in2;
         w.width[0] = w0; w.width[1] = w1; w.width[2] = w2;
-        w.stride[0] = w0; w.stride[1] = w1; w.stride[2] = w2;
-        w.dp = dp; w.dp_stride = J; w.K = w0 + w1 + w2; w.J = J; w.R = rows;
-        w.partial = partial; w.dW = dW; w.db = db;
+        w.stride[0] = s0; w.stride[1] = w1; w.stride[2] = w2;
+        w.dp = dp; w.dp_stride = dp_stride; w.K = w0 + w1 + w2; w.J = J; w.R = rows;
+        w.dW = dW; w.db = db;
         w.chunks = (int)std::max<size_t>(1, std::min<size_t>(kGradChunks, (rows + kRows - 1) / kRows));
-        return weight_grad(w, stream);
+        w.partial = partial;                                  // each job its own stretch
+        partial += (size_t)w.chunks * (w.K + 1) * w.J;
     };
-    for (int dir = 0; dir < 2 && err == cudaSuccess; ++dir) {
+    for (int dir = 0; dir < 2; ++dir) {
         const int Hf = a.f[dir].hidden_dim, Hg = a.g[dir].hidden_dim;
-        err = job(a.H[dir], d, a.X, F, nullptr, 0, a.DFH[dir], Hf, R, a.gf[dir].W1, a.gf[dir].b1);
-        if (err == cudaSuccess) err = job(a.FH[dir], Hf, nullptr, 0, nullptr, 0, a.DPRE_F2[dir], d, R, a.gf[dir].W2, a.gf[dir].b2);
-        if (err == cudaSuccess) err = job(a.Sg[dir], d, nullptr, 0, nullptr, 0, a.DT1[dir], Hg, R, a.gg[dir].W1, a.gg[dir].b1);
-        if (err == cudaSuccess) err = job(a.T1[dir], Hg, nullptr, 0, nullptr, 0, a.DPRE_G2[dir], d, R, a.gg[dir].W2, a.gg[dir].b2);
+        job(a.H[dir], d, d, a.X, F, nullptr, 0, a.DFH[dir], Hf, Hf, R, a.gf[dir].W1, a.gf[dir].b1);
+        job(a.FH[dir], Hf, Hf, nullptr, 0, nullptr, 0, a.DPRE_F2[dir], d, d, R, a.gf[dir].W2, a.gf[dir].b2);
+        job(a.Sg[dir], d, d, nullptr, 0, nullptr, 0, a.DT1[dir], Hg, Hg, R, a.gg[dir].W1, a.gg[dir].b1);
+        job(a.T1[dir], Hg, Hg, nullptr, 0, nullptr, 0, a.DPRE_G2[dir], d, d, R, a.gg[dir].W2, a.gg[dir].b2);
     }
-    for (int i = 0; i < 3 && err == cudaSuccess; ++i) {
-        err = job(a.H[0], d, a.H[1], d, a.X, F, a.DPRE_L[i], d, R, a.gl[i].W1, a.gl[i].b1);
+    for (int i = 0; i < 3; ++i) {
+        job(a.H[0], d, d, a.H[1], d, a.X, F, a.DPRE_L[i], d, d, R, a.gl[i].W1, a.gl[i].b1);
         // h_i: rows are states; the inputs and gradients of set i sit at column offset i * d of [B][3][d]
-        if (err == cudaSuccess) {
-            WeightJob w;
-            w.in[0] = a.Sbuf + i * d; w.in[1] = w.in[2] = nullptr;
-            w.width[0] = d; w.width[1] = w.width[2] = 0;
-            w.stride[0] = 3 * d; w.stride[1] = w.stride[2] = 0;
-            w.dp = a.DPRE_H + i * d; w.dp_stride = 3 * d; w.K = d; w.J = d; w.R = B;
-            w.partial = partial; w.dW = a.gh[i].W1; w.db = a.gh[i].b1;
-            w.chunks = 1;
-            err = weight_grad(w, stream);
-        }
+        job(a.Sbuf + i * d, d, 3 * d, nullptr, 0, nullptr, 0, a.DPRE_H + i * d, 3 * d, d, B, a.gh[i].W1, a.gh[i].b1);
     }
-    if (err == cudaSuccess) err = job(a.Zbuf, Z, nullptr, 0, nullptr, 0, a.DHID, Hh, B, a.ghead.W1, a.ghead.b1);
-    if (err == cudaSuccess) err = job(a.HID, Hh, nullptr, 0, nullptr, 0, a.DLOG, m, B, a.ghead.W2, a.ghead.b2);
-    return err;
+    job(a.Zbuf, Z, Z, nullptr, 0, nullptr, 0, a.DHID, Hh, Hh, B, a.ghead.W1, a.ghead.b1);
+    job(a.HID, Hh, Hh, nullptr, 0, nullptr, 0, a.DLOG, m, m, B, a.ghead.W2, a.ghead.b2);
+    err = weight_grads(by_row, stream);
+    if (err != cudaSuccess) return err;
+    return weight_grads(by_state, stream);
 }
 
 }  // namespace placeto
