@@ -91,17 +91,17 @@ embed_rounds_d32_kernel(const EmbedArgs a, const float *__restrict__ Min0,
         __syncthreads();
     }
     const int ppn = (B + 1) >> 1;                       // state pairs per node
-    const long long items = (long long)n * ppn;
-    const long long step = (long long)gridDim.x * kWarps;
+    const int items = n * ppn;                          // n * B < 2^31 is checked by the caller
+    const int step = gridDim.x * kWarps;
     struct Pass {
         int pos, v, e0, e1, b0, b1;
         bool two;
         float x0, x1, t[kAhead][2];
     };
     // issues the loads of one pass: features and the first kAhead neighbour rows
-    auto fetch = [&](long long item, Pass &p) {
-        p.pos = (int)(item / ppn);
-        p.b0 = (int)(item - (long long)p.pos * ppn) * 2;
+    auto fetch = [&](int item, Pass &p) {
+        p.pos = (int)((unsigned)item / (unsigned)ppn);
+        p.b0 = (item - p.pos * ppn) * 2;
         p.two = p.b0 + 1 < B;
         p.b1 = p.two ? p.b0 + 1 : p.b0;
         p.v = order[p.pos];
@@ -120,7 +120,7 @@ embed_rounds_d32_kernel(const EmbedArgs a, const float *__restrict__ Min0,
             }
         }
     };
-    long long item = (long long)blockIdx.x * kWarps + warp;
+    int item = blockIdx.x * kWarps + warp;
     Pass cur, nxt;
     if (item < items) fetch(item, cur);
     for (; item < items; item += step) {
