@@ -407,21 +407,29 @@ __global__ void __launch_bounds__(kThreads)
 grad_weight_partial_kernel(const WeightJobs jobs) {
     extern __shared__ __align__(16) float smem[];
     const WeightJob &w = jobs.job[blockIdx.z];
-    if ((int)blockIdx.x >= w.chunks || (int)blockIdx.y * 1024 >= (w.K + 1) * w.J) return;
     const int K = w.K, J = w.J;
-    float *in = smem;                  // [kRows][K + 1] (last column = 1 for the bias)
-    float *dp = in + kRows * (K + 1);  // [kRows][J]
+    const int Kp = (K + 1 + 3) & ~3, Jp = (J + 3) & ~3;      // padded with zeros to whole 4 x 4 tiles
+    const int tiles_j = Jp >> 2, n_tiles = (Kp >> 2) * tiles_j;
+    if ((int)blockIdx.x >= w.chunks || (int)blockIdx.y * kThreads >= n_tiles) return;
+    float *in = smem;                  // [kRows][Kp] (column K = 1 for the bias)
+    float *dp = in + kRows * Kp;       // [kRows][Jp]
     const int chunk = blockIdx.x;
     const size_t per = (w.R + w.chunks - 1) / w.chunks;
     const size_t r_begin = (size_t)chunk * per, r_end = min(w.R, r_begin + per);
-    const int tile0 = blockIdx.y * 1024;                 // output elements [tile0, tile0 + 1024)
-    const int n_out = (K + 1) * J;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};                 // elements tile0 + threadIdx.x + 256 q
+    // a thread owns one 4 x 4 tile of the product: two 128-bit shared loads feed 16 FMAs
+    const int tile = blockIdx.y * kThreads + threadIdx.x;
+    const bool live = tile < n_tiles;
+    const int tk = live ? tile / tiles_j : 0, tj = live ? tile - tk * tiles_j : 0;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
     for (size_t r0 = r_begin; r0 < r_end; r0 += kRows) {
         const int rows = (int)min((size_t)kRows, r_end - r0);
-        for (int i = threadIdx.x; i < rows * (K + 1); i += kThreads) {
-            const int r = i / (K + 1), k = i - r * (K + 1);
-            float v = 1.f;
+        for (int i = threadIdx.x; i < rows * Kp; i += kThreads) {
+            const int r = i / Kp, k = i - r * Kp;
+            float v = k == K ? 1.f : 0.f;
             if (k < K) {
                 int kk = k, part = 0;
                 while (kk >= w.width[part]) { kk -= w.width[part]; ++part; }
@@ -429,27 +437,34 @@ grad_weight_partial_kernel(const WeightJobs jobs) {
             }
             in[i] = v;
         }
-        for (int i = threadIdx.x; i < rows * J; i += kThreads) {
-            const int r = i / J, j = i - r * J;
-            dp[i] = w.dp[(r0 + r) * w.dp_stride + j];
+        for (int i = threadIdx.x; i < rows * Jp; i += kThreads) {
+            const int r = i / Jp, j = i - r * Jp;
+            dp[i] = j < J ? w.dp[(r0 + r) * w.dp_stride + j] : 0.f;
         }
         __syncthreads();
+        if (live) {
+            const float *pa = in + 4 * tk, *pb = dp + 4 * tj;
+            for (int r = 0; r < rows; ++r) {
+                const float4 x = *reinterpret_cast<const float4 *>(pa + r * Kp);
+                const float4 y = *reinterpret_cast<const float4 *>(pb + r * Jp);
+                const float xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int o = tile0 + threadIdx.x + kThreads * q;
-            if (o < n_out) {
-                const int k = o / J, j = o - k * J;
-                float s = acc[q];
-                for (int r = 0; r < rows; ++r) s = fmaf(in[r * (K + 1) + k], dp[r * J + j], s);
-                acc[q] = s;
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xs[i], ys[j], acc[i][j]);
             }
         }
         __syncthreads();
     }
+    if (live) {
+        const int n_out = (K + 1) * J;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const int o = tile0 + threadIdx.x + kThreads * q;
-        if (o < n_out) w.partial[(size_t)chunk * n_out + o] = acc[q];
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int k = 4 * tk + i, jj = 4 * tj + j;
+                if (k <= K && jj < J) w.partial[(size_t)chunk * n_out + k * J + jj] = acc[i][j];
+            }
     }
 }
 
@@ -480,17 +495,19 @@ grad_weight_reduce_kernel(const WeightJobs jobs) {
 cudaError_t weight_grads(const WeightJobs &jobs, cudaStream_t stream) {
     if (jobs.count == 0) return cudaSuccess;
     size_t smem = 0;
-    int max_chunks = 1, max_out = 1;
+    int max_chunks = 1, max_out = 1, max_tiles = 1;
     for (int i = 0; i < jobs.count; ++i) {
         const WeightJob &w = jobs.job[i];
-        smem = std::max(smem, ((size_t)kRows * (w.K + 1) + (size_t)kRows * w.J) * sizeof(float));
+        const int Kp = (w.K + 1 + 3) & ~3, Jp = (w.J + 3) & ~3;
+        smem = std::max(smem, (size_t)kRows * (Kp + Jp) * sizeof(float));
         max_chunks = std::max(max_chunks, w.chunks);
         max_out = std::max(max_out, (w.K + 1) * w.J);
+        max_tiles = std::max(max_tiles, (Kp / 4) * (Jp / 4));
     }
     cudaError_t err = cudaFuncSetAttribute(grad_weight_partial_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    grad_weight_partial_kernel<<<dim3(max_chunks, (max_out + 1023) / 1024, jobs.count), kThreads, smem, stream>>>(jobs);
+    grad_weight_partial_kernel<<<dim3(max_chunks, (max_tiles + kThreads - 1) / kThreads, jobs.count), kThreads, smem, stream>>>(jobs);
     count_launch();
     grad_weight_reduce_kernel<<<dim3((max_out + 31) / 32, jobs.count), 256, 0, stream>>>(jobs);
     count_launch();
