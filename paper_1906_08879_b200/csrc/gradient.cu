@@ -257,7 +257,59 @@ grad_head_kernel(const GradArgs a) {
 }
 
 // ------------------------------------------------------------------ 3. sweeps
-// One block per (state slice, direction): levels in reverse order.
+constexpr int kSweepRows = 64;     // rows per pass of the sweep kernel
+
+// out(r, j) = sum_k A[r][k] W[k][j] for rows x J outputs, all operands in shared
+// memory (A row stride lda, odd; W row stride ldw, a multiple of 4). A thread owns
+// tiles of 2 rows x 4 columns: two scalar loads and one 128-bit load feed 8 FMAs.
+template <typename Epilogue>
+__device__ __forceinline__ void tile_product(const float *A, int lda, const float *W, int ldw, int K,
+                                             int J, int rows, Epilogue done) {
+    if (rows * J <= 2 * kThreads) {
+        // a short pass (narrow level, few states): one output per thread keeps the chain short
+        for (int i = threadIdx.x; i < rows * J; i += kThreads) {
+            const int r = i / J, j = i - r * J;
+            const float *x = A + r * lda, *w = W + j;
+            float c = 0.f, e = 0.f;
+            int k = 0;
+            for (; k + 2 <= K; k += 2) {
+                c = fmaf(x[k], w[k * ldw], c);
+                e = fmaf(x[k + 1], w[(k + 1) * ldw], e);
+            }
+            if (k < K) c = fmaf(x[k], w[k * ldw], c);
+            done(r, j, c + e);
+        }
+        return;
+    }
+    const int tiles_j = (J + 3) >> 2, tiles_r = (rows + 1) >> 1;
+    for (int tile = threadIdx.x; tile < tiles_r * tiles_j; tile += kThreads) {
+        const int tr = tile / tiles_j, tj = tile - tr * tiles_j;
+        const int r0 = 2 * tr, r1 = min(r0 + 1, rows - 1);
+        const float *a0 = A + r0 * lda, *a1 = A + r1 * lda, *w = W + 4 * tj;
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int k = 0; k < K; ++k) {
+            const float4 wv = *reinterpret_cast<const float4 *>(w + k * ldw);
+            const float x0 = a0[k], x1 = a1[k];
+            c0[0] = fmaf(x0, wv.x, c0[0]); c0[1] = fmaf(x0, wv.y, c0[1]);
+            c0[2] = fmaf(x0, wv.z, c0[2]); c0[3] = fmaf(x0, wv.w, c0[3]);
+            c1[0] = fmaf(x1, wv.x, c1[0]); c1[1] = fmaf(x1, wv.y, c1[1]);
+            c1[2] = fmaf(x1, wv.z, c1[2]); c1[3] = fmaf(x1, wv.w, c1[3]);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int j = 4 * tj + q;
+            if (j < J) {
+                done(r0, j, c0[q]);
+                if (r0 + 1 < rows) done(r0 + 1, j, c1[q]);
+            }
+        }
+    }
+}
+
+// One block per (state slice, direction): levels in reverse order. Per pass of up
+// to kSweepRows rows: one phase brings everything the pass needs from global
+// memory into shared memory (so a level pays one memory latency, not one per
+// step), then four shared-memory products push the gradient through f and g.
 __global__ void __launch_bounds__(kThreads)
 grad_sweep_kernel(const GradArgs a, int S) {
     extern __shared__ __align__(16) float smem[];
@@ -269,110 +321,107 @@ grad_sweep_kernel(const GradArgs a, int S) {
     // consumers of a node's message: children for the top-down pass, parents for the bottom-up one
     const int *cons_ptr = dir == 0 ? a.child_ptr : a.parent_ptr;
     const int *cons = dir == 0 ? a.child : a.parent;
-    const int W = max(max(d, Hf), Hg);
-    float *bufA = smem, *bufB = smem + kRows * W, *bufC = bufB + kRows * W;   // [kRows][W] each
-    // the direction's matrices in shared memory, rows padded by one float so that
-    // both the row-wise and the column-wise reads below are free of bank conflicts
-    const int sf = Hf + 1, sd = d + 1, sg = Hg + 1;
-    float *wf1 = bufC + kRows * W;         // [d][Hf]: the h rows of f's first layer
-    float *wf2 = wf1 + d * sf;             // [Hf][d]
-    float *wg1 = wf2 + Hf * sd;            // [d][Hg]
-    float *wg2 = wg1 + d * sg;             // [Hg][d]
-    float *bg1 = wg2 + Hg * sd;            // [Hg]
-    for (int i = threadIdx.x; i < d * Hf; i += kThreads) wf1[(i / Hf) * sf + i % Hf] = f.W1[i];
-    for (int i = threadIdx.x; i < Hf * d; i += kThreads) wf2[(i / d) * sd + i % d] = f.W2[i];
-    for (int i = threadIdx.x; i < d * Hg; i += kThreads) wg1[(i / Hg) * sg + i % Hg] = gm.W1[i];
-    for (int i = threadIdx.x; i < Hg * d; i += kThreads) wg2[(i / d) * sd + i % d] = gm.W2[i];
+    const int W = max(max(d, Hf), Hg) | 1;         // odd row stride of the row buffers
+    float *bufA = smem;                            // [rows][W] dpre_f2, later dt1
+    float *bufB = bufA + kSweepRows * W;           // dfh
+    float *bufC = bufB + kSweepRows * W;           // dpre_g2
+    float *bufD = bufC + kSweepRows * W;           // d/dh from the pooling
+    float *bufS = bufD + kSweepRows * W;           // summed neighbour messages
+    float *mskF = bufS + kSweepRows * W;           // fh > 0
+    float *mskH = mskF + kSweepRows * W;           // h > 0
+    // the direction's matrices, each in the orientation its product reads row-wise
+    const int pd = (d + 3) & ~3, pf = (Hf + 3) & ~3, pg = (Hg + 3) & ~3;
+    float *wf2t = mskH + kSweepRows * W;           // [d][pf]:  W_f2^T
+    float *wf1t = wf2t + d * pf;                   // [Hf][pd]: (h rows of W_f1)^T
+    float *wg1 = wf1t + Hf * pd;                   // [d][pg]:  W_g1
+    float *wg2t = wg1 + d * pg;                    // [d][pg]:  W_g2^T
+    float *wg1t = wg2t + d * pg;                   // [Hg][pd]: W_g1^T
+    float *bg1 = wg1t + Hg * pd;                   // [Hg]
+    for (int i = threadIdx.x; i < Hf * d; i += kThreads) { const int k = i / d, j = i - k * d; wf2t[j * pf + k] = f.W2[i]; }
+    for (int i = threadIdx.x; i < d * Hf; i += kThreads) { const int j = i / Hf, k = i - j * Hf; wf1t[k * pd + j] = f.W1[i]; }
+    for (int i = threadIdx.x; i < d * Hg; i += kThreads) { const int j = i / Hg, k = i - j * Hg; wg1[j * pg + k] = gm.W1[i]; wg1t[k * pd + j] = gm.W1[i]; }
+    for (int i = threadIdx.x; i < Hg * d; i += kThreads) { const int k = i / d, j = i - k * d; wg2t[j * pg + k] = gm.W2[i]; }
     for (int i = threadIdx.x; i < Hg; i += kThreads) bg1[i] = gm.b1[i];
     __syncthreads();
     const float *H = a.H[dir], *M = a.M[dir], *FH = a.FH[dir];
     for (int level = lv.n_levels - 1; level >= 0; --level) {
         const int p0 = lv.level_ptr[level], width = lv.level_ptr[level + 1] - p0;
         const int total = width * nb;
-        for (int r0 = 0; r0 < total; r0 += kRows) {
-            const int rows = min(kRows, total - r0);
+        for (int r0 = 0; r0 < total; r0 += kSweepRows) {
+            const int rows = min(kSweepRows, total - r0);
             auto row_of = [&](int r, int &pos, size_t &off) {
                 const int q = (r0 + r) / nb;
                 pos = p0 + q;
                 off = (size_t)lv.order[pos] * B + b0 + (r0 + r - q * nb);
             };
-            // dpre_f2 = (sum over consumers of ds) * (m > 0)          -> bufA [rows][d]
+            // ---- everything the pass reads from global memory
             for (int i = threadIdx.x; i < rows * d; i += kThreads) {
                 const int r = i / d, j = i - r * d;
                 int pos; size_t off;
                 row_of(r, pos, off);
                 const int u = lv.order[pos];
                 const int b = (int)(off - (size_t)u * B);
-                float acc = 0.f;
+                float dm = 0.f, s = 0.f;
                 for (int e = cons_ptr[u]; e < cons_ptr[u + 1]; ++e)
-                    acc += a.DS[dir][((size_t)cons[e] * B + b) * d + j];
-                acc = M[off * d + j] > 0.f ? acc : 0.f;
-                bufA[r * W + j] = acc;
-                a.DPRE_F2[dir][off * d + j] = acc;
+                    dm += a.DS[dir][((size_t)cons[e] * B + b) * d + j];
+                for (int e = lv.nbr_ptr[pos]; e < lv.nbr_ptr[pos + 1]; ++e)
+                    s += M[((size_t)lv.nbr[e] * B + b) * d + j];
+                dm = M[off * d + j] > 0.f ? dm : 0.f;            // dpre_f2
+                bufA[r * W + j] = dm;
+                a.DPRE_F2[dir][off * d + j] = dm;
+                bufS[r * W + j] = s;
+                a.Sg[dir][off * d + j] = s;
+                bufD[r * W + j] = a.DH[dir][off * d + j];
+                mskH[r * W + j] = H[off * d + j] > 0.f ? 1.f : 0.f;
             }
-            __syncthreads();
-            // dfh = (dpre_f2 W_f2^T) * (fh > 0)                        -> bufB [rows][Hf]
             for (int i = threadIdx.x; i < rows * Hf; i += kThreads) {
                 const int r = i / Hf, k = i - r * Hf;
                 int pos; size_t off;
                 row_of(r, pos, off);
-                float acc = 0.f;
-                for (int j = 0; j < d; ++j) acc = fmaf(bufA[r * W + j], wf2[k * sd + j], acc);
-                acc = FH[off * Hf + k] > 0.f ? acc : 0.f;
-                bufB[r * W + k] = acc;
-                a.DFH[dir][off * Hf + k] = acc;
+                mskF[r * W + k] = FH[off * Hf + k] > 0.f ? 1.f : 0.f;
             }
             __syncthreads();
-            // dh = dH_pool + dfh W_f1[0:d]^T ; dpre_g2 = dh * (h > 0)  -> bufA [rows][d]
-            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
-                const int r = i / d, j = i - r * d;
+            // ---- dfh = (dpre_f2 W_f2^T) * (fh > 0)
+            tile_product(bufA, W, wf2t, pf, d, Hf, rows, [&](int r, int k, float v) {
                 int pos; size_t off;
                 row_of(r, pos, off);
-                float acc = a.DH[dir][off * d + j];
-                for (int k = 0; k < Hf; ++k) acc = fmaf(bufB[r * W + k], wf1[j * sf + k], acc);
-                acc = H[off * d + j] > 0.f ? acc : 0.f;
-                a.DPRE_G2[dir][off * d + j] = acc;
-                bufC[r * W + j] = acc;
-            }
-            // s = sum of the neighbours' messages                       -> bufB [rows][d] (after the reads above)
+                v *= mskF[r * W + k];
+                bufB[r * W + k] = v;
+                a.DFH[dir][off * Hf + k] = v;
+            });
             __syncthreads();
-            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
-                const int r = i / d, j = i - r * d;
+            // ---- dpre_g2 = (dH_pool + dfh W_f1[0:d]^T) * (h > 0)
+            tile_product(bufB, W, wf1t, pd, Hf, d, rows, [&](int r, int j, float v) {
                 int pos; size_t off;
                 row_of(r, pos, off);
-                const int b = (int)(off - (size_t)lv.order[pos] * B);
-                float acc = 0.f;
-                for (int e = lv.nbr_ptr[pos]; e < lv.nbr_ptr[pos + 1]; ++e)
-                    acc += M[((size_t)lv.nbr[e] * B + b) * d + j];
-                bufB[r * W + j] = acc;
-                a.Sg[dir][off * d + j] = acc;
-            }
+                v = (v + bufD[r * W + j]) * mskH[r * W + j];
+                bufC[r * W + j] = v;
+                a.DPRE_G2[dir][off * d + j] = v;
+            });
             __syncthreads();
-            // t1 = relu(s W_g1 + b) ; dt1 = (dpre_g2 W_g2^T) * (t1 > 0) -> bufA [rows][Hg]
-            for (int i = threadIdx.x; i < rows * Hg; i += kThreads) {
-                const int r = i / Hg, k = i - r * Hg;
+            // ---- t1 = relu(s W_g1 + b), dt1 = (dpre_g2 W_g2^T) * (t1 > 0): t1 first, into bufA as a mask
+            tile_product(bufS, W, wg1, pg, d, Hg, rows, [&](int r, int k, float v) {
                 int pos; size_t off;
                 row_of(r, pos, off);
-                float t1 = bg1[k];
-                for (int j = 0; j < d; ++j) t1 = fmaf(bufB[r * W + j], wg1[j * sg + k], t1);
-                t1 = fmaxf(t1, 0.f);
-                float acc = 0.f;
-                for (int j = 0; j < d; ++j) acc = fmaf(bufC[r * W + j], wg2[k * sd + j], acc);
-                acc = t1 > 0.f ? acc : 0.f;
-                a.T1[dir][off * Hg + k] = t1;
-                a.DT1[dir][off * Hg + k] = acc;
-                bufA[r * W + k] = acc;
-            }
+                v = fmaxf(v + bg1[k], 0.f);
+                a.T1[dir][off * Hg + k] = v;
+                bufA[r * W + k] = v > 0.f ? 1.f : 0.f;
+            });
             __syncthreads();
-            // ds = dt1 W_g1^T                                            -> DS
-            for (int i = threadIdx.x; i < rows * d; i += kThreads) {
-                const int r = i / d, j = i - r * d;
+            tile_product(bufC, W, wg2t, pg, d, Hg, rows, [&](int r, int k, float v) {
                 int pos; size_t off;
                 row_of(r, pos, off);
-                float acc = 0.f;
-                for (int k = 0; k < Hg; ++k) acc = fmaf(bufA[r * W + k], wg1[j * sg + k], acc);
-                a.DS[dir][off * d + j] = acc;
-            }
+                v *= bufA[r * W + k];
+                a.DT1[dir][off * Hg + k] = v;
+                bufB[r * W + k] = v;
+            });
+            __syncthreads();
+            // ---- ds = dt1 W_g1^T
+            tile_product(bufB, W, wg1t, pd, Hg, d, rows, [&](int r, int j, float v) {
+                int pos; size_t off;
+                row_of(r, pos, off);
+                a.DS[dir][off * d + j] = v;
+            });
             __syncthreads();
         }
         __threadfence_block();
@@ -590,9 +639,11 @@ cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, 
         size_t wfloats = 0;
         for (int dir = 0; dir < 2; ++dir) {
             const size_t Hf = a.f[dir].hidden_dim, Hg = a.g[dir].hidden_dim;
-            wfloats = std::max(wfloats, d * (Hf + 1) + Hf * ((size_t)d + 1) + d * (Hg + 1) + Hg * ((size_t)d + 1) + Hg);
+            const size_t pd = ((size_t)d + 3) & ~size_t(3), pf = (Hf + 3) & ~size_t(3), pg = (Hg + 3) & ~size_t(3);
+            wfloats = std::max(wfloats, d * pf + Hf * pd + 2 * d * pg + Hg * pd + Hg);
         }
-        const size_t smem = (3 * (size_t)kRows * W + wfloats) * sizeof(float);
+        W |= 1;
+        const size_t smem = (7 * (size_t)kSweepRows * W + wfloats) * sizeof(float);
         if (smem > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
         err = cudaFuncSetAttribute(grad_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
