@@ -30,18 +30,37 @@ struct Pool32Plan {
     size_t smem_bytes;
 };
 
+typedef unsigned long long pair_t;   // two FP32 values in one 64-bit register pair
+
+__device__ __forceinline__ pair_t pack2(float lo, float hi) {
+    pair_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ float sum2(pair_t v) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+// two independent FP32 FMAs in one instruction (sm_100 packed arithmetic)
+__device__ __forceinline__ pair_t fma2(pair_t a, pair_t b, pair_t c) {
+    pair_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// acc[r] += in[r][0..K) . w for R rows; w holds the column as pairs (w[2i], w[2i+1]),
+// every 128-bit shared load feeds two packed FMAs.
 template <int R, int K>
-__device__ __forceinline__ void fma_rows(const float *w, const float *const (&in)[R],
-                                         float (&acc)[R][2]) {
+__device__ __forceinline__ void fma_rows(const pair_t *w, const float *const (&in)[R],
+                                         pair_t (&acc)[R][2]) {
 #pragma unroll
     for (int k = 0; k < K; k += 4) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const float4 u = *reinterpret_cast<const float4 *>(in[r] + k);
-            acc[r][0] = fmaf(u.x, w[k], acc[r][0]);
-            acc[r][1] = fmaf(u.y, w[k + 1], acc[r][1]);
-            acc[r][0] = fmaf(u.z, w[k + 2], acc[r][0]);
-            acc[r][1] = fmaf(u.w, w[k + 3], acc[r][1]);
+            const ulonglong2 u = *reinterpret_cast<const ulonglong2 *>(in[r] + k);
+            acc[r][0] = fma2(u.x, w[k / 2], acc[r][0]);
+            acc[r][1] = fma2(u.y, w[k / 2 + 1], acc[r][1]);
         }
     }
 }
@@ -102,9 +121,10 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     const uint8_t *rel = a.relation + (size_t)(valid ? c : 0) * n + u0;
     float *out = a.partial + ((size_t)chunk * B + b) * 3 * kD;
     for (int i = 0; i < 3; ++i) {
-        float w[E];
+        pair_t w[E / 2];
 #pragma unroll
-        for (int k = 0; k < E; ++k) w[k] = Ws[(i * E + k) * kD + lane];
+        for (int k = 0; k < E; k += 2)
+            w[k / 2] = pack2(Ws[(i * E + k) * kD + lane], Ws[(i * E + k + 1) * kD + lane]);
         const float bias = bs[i * kD + lane];
         float total = 0.f;
         for (int base = 0; base < nu && valid; base += 32) {
@@ -116,26 +136,26 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
                 if (mask) {
                     const int qb = base + __ffs(mask) - 1;
                     mask &= mask - 1;
-                    float acc[2][2] = {{bias, 0.f}, {bias, 0.f}};
+                    pair_t acc[2][2] = {{pack2(bias, 0.f), 0ull}, {pack2(bias, 0.f), 0ull}};
                     const size_t ra = (size_t)qa * kWarps + warp, rb = (size_t)qb * kWarps + warp;
                     const float *const pd[2] = {hd + ra * kD, hd + rb * kD};
                     const float *const pu[2] = {hu + ra * kD, hu + rb * kD};
                     const float *const px[2] = {xs + ra * FP, xs + rb * FP};
                     fma_rows<2, kD>(w, pd, acc);
-                    fma_rows<2, kD>(w + kD, pu, acc);
-                    fma_rows<2, FP>(w + 2 * kD, px, acc);
-                    total += fmaxf(acc[0][0] + acc[0][1], 0.f);
-                    total += fmaxf(acc[1][0] + acc[1][1], 0.f);
+                    fma_rows<2, kD>(w + kD / 2, pu, acc);
+                    fma_rows<2, FP>(w + kD, px, acc);
+                    total += fmaxf(sum2(acc[0][0]) + sum2(acc[0][1]), 0.f);
+                    total += fmaxf(sum2(acc[1][0]) + sum2(acc[1][1]), 0.f);
                 } else {
-                    float acc[1][2] = {{bias, 0.f}};
+                    pair_t acc[1][2] = {{pack2(bias, 0.f), 0ull}};
                     const size_t ra = (size_t)qa * kWarps + warp;
                     const float *const pd[1] = {hd + ra * kD};
                     const float *const pu[1] = {hu + ra * kD};
                     const float *const px[1] = {xs + ra * FP};
                     fma_rows<1, kD>(w, pd, acc);
-                    fma_rows<1, kD>(w + kD, pu, acc);
-                    fma_rows<1, FP>(w + 2 * kD, px, acc);
-                    total += fmaxf(acc[0][0] + acc[0][1], 0.f);
+                    fma_rows<1, kD>(w + kD / 2, pu, acc);
+                    fma_rows<1, FP>(w + kD, px, acc);
+                    total += fmaxf(sum2(acc[0][0]) + sum2(acc[0][1]), 0.f);
                 }
             }
         }
