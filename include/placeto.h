@@ -332,17 +332,20 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
  * cur, actions    : DEVICE int32[B] (actions < m; a state whose cur is outside [0, n)
  *                   contributes nothing).      advantages : DEVICE float[B].
  * grads           : a placeto_weights of the same shapes as w whose pointers address
- *                   writable DEVICE buffers; every array is overwritten with dJ/d(array).
+ *                   writable DEVICE buffers; every array is overwritten with dJ/d(array), or,
+ *                   with PLACETO_GRAD_ACCUMULATE in flags, has dJ/d(array) added to it (a large
+ *                   set of states can then be differentiated in several calls).
  * workspace       : DEVICE, at least placeto_workspace_bytes(.., PLACETO_CALL_GRADIENT, 0):
  *                   about 2 * n * B * (2 * (hidden_f + hidden_g) + 6 d) + 3 n B d floats.
  * Shapes: two-layer ReLU f and g, single-layer ReLU l_i and h_i, two-layer head with a
  * ReLU hidden layer and a linear output; otherwise PLACETO_ERR_UNSUPPORTED.
  */
+#define PLACETO_GRAD_ACCUMULATE 1u
 placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_weights *w, const float *X,
                                        const float *H_down, const float *H_up, const int32_t *cur,
                                        const int32_t *actions, const float *advantages, float beta,
                                        int32_t B, const placeto_weights *grads, void *workspace,
-                                       size_t workspace_bytes, void *stream);
+                                       size_t workspace_bytes, uint32_t flags, void *stream);
 
 /*
  * placeto_policy_logits without a workspace argument, for callers that must not

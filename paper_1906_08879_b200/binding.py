@@ -389,15 +389,17 @@ def zero_gradients(weights: dict, device="cuda") -> "Weights":
 
 
 def placeto_policy_gradient(g: Graph, w: Weights, X, H_down, H_up, cur, actions, advantages,
-                            beta: float, grads: Weights, ws=None, stream=None):
-    """dJ/d(weights) into `grads` (a Weights of the same shapes, see zero_gradients)."""
+                            beta: float, grads: Weights, ws=None, stream=None, accumulate: bool = False):
+    """dJ/d(weights) into `grads` (a Weights of the same shapes, see zero_gradients);
+    with `accumulate` it is added to what `grads` holds."""
     B = X.shape[1]
     if ws is None:
         ws = workspace(g, w, B, CALL_GRADIENT, 0, X.device)
     _check(_lib.placeto_policy_gradient(g.handle, ctypes.byref(w.c), _p(X), _p(H_down), _p(H_up), _p(cur),
                                         _p(actions), _p(advantages), ctypes.c_float(beta),
                                         ctypes.c_int32(B), ctypes.byref(grads.c), _p(ws),
-                                        ctypes.c_size_t(ws.numel()), _stream(stream)),
+                                        ctypes.c_size_t(ws.numel()), ctypes.c_uint32(1 if accumulate else 0),
+                                        _stream(stream)),
            "placeto_policy_gradient")
     return grads
 

@@ -683,8 +683,9 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
                                        const float *H_down, const float *H_up, const int32_t *cur,
                                        const int32_t *actions, const float *advantages, float beta,
                                        int32_t B, const placeto_weights *grads, void *workspace,
-                                       size_t workspace_bytes, void *stream) {
+                                       size_t workspace_bytes, uint32_t flags, void *stream) {
     t_launches = 0;
+    if (flags & ~PLACETO_GRAD_ACCUMULATE) return PLACETO_ERR_INVALID_ARG;
     if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
     placeto_status s = embed_weights_ok(w);
     if (s == PLACETO_OK) s = pool_weights_ok(w);
@@ -726,6 +727,7 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
     if (!policy_gradient_applicable(a)) return PLACETO_ERR_UNSUPPORTED;
     a.X = X; a.H[0] = H_down; a.H[1] = H_up;
     a.cur = cur; a.actions = actions; a.advantages = advantages; a.beta = beta;
+    a.accumulate = (flags & PLACETO_GRAD_ACCUMULATE) ? 1 : 0;
     auto out = [](const placeto_mlp &m) {
         GradOut o;
         o.W1 = const_cast<float *>(m.W1); o.b1 = const_cast<float *>(m.b1);

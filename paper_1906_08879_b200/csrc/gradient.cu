@@ -442,6 +442,7 @@ struct WeightJob {
     float *partial;       // [chunks][(K + 1) * J], row K holds the bias sums
     float *dW, *db;
     int chunks;
+    int accumulate;       // 1: add to what dW, db hold instead of overwriting
 };
 
 constexpr int kMaxJobs = 16;
@@ -536,8 +537,8 @@ grad_weight_reduce_kernel(const WeightJobs jobs) {
         float total = 0.f;
 #pragma unroll
         for (int q = 0; q < 8; ++q) total += sums[q][lane];
-        if (o < w.K * w.J) w.dW[o] = total;
-        else w.db[o - w.K * w.J] = total;
+        float *dst = o < w.K * w.J ? w.dW + o : w.db + (o - w.K * w.J);
+        *dst = w.accumulate ? *dst + total : total;
     }
 }
 
@@ -666,6 +667,7 @@ cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, 
         w.stride[0] = s0; w.stride[1] = w1; w.stride[2] = w2;
         w.dp = dp; w.dp_stride = dp_stride; w.K = w0 + w1 + w2; w.J = J; w.R = rows;
         w.dW = dW; w.db = db;
+        w.accumulate = a.accumulate;
         w.chunks = (int)std::max<size_t>(1, std::min<size_t>(kGradChunks, (rows + kRows - 1) / kRows));
         w.partial = partial;                                  // each job its own stretch
         partial += (size_t)w.chunks * (w.K + 1) * w.J;

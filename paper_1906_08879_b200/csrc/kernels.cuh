@@ -101,6 +101,7 @@ struct GradArgs {
     const int *cur, *actions;
     const float *advantages;
     float beta;
+    int accumulate;            // 1: gradients are added to the output buffers
     float *FH[2], *DFH[2], *T1[2], *DT1[2], *M[2], *DS[2], *DPRE_F2[2], *DPRE_G2[2], *Sg[2], *DH[2];
     float *DPRE_L[3], *Zbuf, *HID, *DHID, *DLOG, *Sbuf, *DPRE_H;
     GradOut gf[2], gg[2], gl[3], gh[3], ghead;

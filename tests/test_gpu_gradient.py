@@ -92,6 +92,23 @@ def test_inception_shaped_graph():
     compare(cfg, grads, gradient.gradient(cfg, actions, adv, 0.05))
 
 
+def test_accumulating_over_two_halves_of_the_batch():
+    cfg, actions, adv = small_case(12, n=16, m=4, d=32, B=24)
+    adv = adv.astype(np.float32).astype(np.float64)
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    grads = placeto.binding.zero_gradients(cfg["weights"])
+    for k, sel in enumerate((slice(0, 10), slice(10, 24))):
+        cur = dev_t(cfg["cur"][sel])
+        X = placeto.placeto_build_features(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"][sel]),
+                                           cur, dev_t(cfg["placed"][sel]), cfg["m"])
+        Hd, Hu = placeto.placeto_embed_forward(g, w, X)
+        placeto.placeto_policy_gradient(g, w, X, Hd, Hu, cur, dev_t(actions[sel].astype(np.int32)),
+                                        dev_t(adv[sel].astype(np.float32)), 0.2, grads, accumulate=k > 0)
+    torch.cuda.synchronize()
+    compare(cfg, grads, gradient.gradient(cfg, actions, adv, 0.2))
+
+
 def test_reproducible_and_unsupported_shapes():
     cfg, actions, adv = small_case(3, n=14, m=4, d=32, B=17)
     a = gpu_gradient(cfg, actions, adv, 0.1)
