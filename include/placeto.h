@@ -54,7 +54,7 @@ typedef enum {
                                      placeto_policy_logits_static */
 } placeto_status;
 
-/* Limits of this build. */
+/* Limits of the library. */
 #define PLACETO_MAX_D 128      /* embedding width d */
 #define PLACETO_MAX_F 64       /* feature width F */
 #define PLACETO_MAX_M 60       /* devices m (F = m + 4 in build_features) */
