@@ -228,10 +228,14 @@ placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weig
                                       size_t workspace_bytes, uint32_t flags, void *stream);
 
 /*
- * Whole path from HOST state arrays to HOST results: copies cost, bytes, dev, cur,
- * placed to the device (cudaMemcpyAsync on `stream`; pinned host memory makes them
- * truly asynchronous), runs the path, copies logits (and probs unless NULL) back and
- * waits for the stream before returning. Weights and workspace stay DEVICE pointers.
+ * Whole path from HOST state arrays to HOST results: brings cost, bytes, dev, cur,
+ * placed to the device, runs the path, returns logits (and probs unless NULL) to the
+ * host and waits for the stream before returning. When all five inputs are page-locked
+ * host memory (cudaHostAlloc, cudaHostRegister, a pinned torch tensor) one kernel
+ * gathers them across the host link, and when the outputs are page-locked too the
+ * head kernel writes them in place; pageable buffers are moved with cudaMemcpyAsync
+ * on `stream` instead. Either way the same bytes cross the link once per call.
+ * Weights and workspace stay DEVICE pointers.
  */
 placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto_weights *w,
                                            const float *cost, const float *bytes,

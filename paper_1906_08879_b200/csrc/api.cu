@@ -152,6 +152,17 @@ bool flags_ok(uint32_t flags) {
     return (sched & (sched - 1)) == 0;   // at most one schedule
 }
 
+// The device-side address of a page-locked (cudaHostAlloc / cudaHostRegister) host
+// buffer, or nullptr when the pointer is pageable host memory or anything else.
+const void *device_alias(const void *p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 placeto_status cuda_status(cudaError_t e) {
     if (e == cudaSuccess) return PLACETO_OK;
     if (e == cudaErrorCooperativeLaunchTooLarge) return PLACETO_ERR_UNSUPPORTED;
@@ -521,12 +532,28 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     float *d_logits = reinterpret_cast<float *>(ws + L.logits);
     float *d_probs = reinterpret_cast<float *>(ws + L.probs);
     const size_t mB = (size_t)B * w->m * sizeof(float);
-    if (cudaMemcpyAsync(d_cost, cost, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(d_bytes, bytes, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(d_dev, dev, n * B, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(d_placed, placed, n * B, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(d_cur, cur, (size_t)B * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return PLACETO_ERR_CUDA;
+    // Page-locked host buffers are addressable from the device: the five inputs are
+    // then gathered by one kernel instead of five copies, and the head kernel writes
+    // logits and probabilities straight into the caller's buffers. Pageable buffers
+    // take the copy path.
+    const void *src[5] = {cost, bytes, dev, placed, cur};
+    void *dst[5] = {d_cost, d_bytes, d_dev, d_placed, d_cur};
+    const size_t len[5] = {n * sizeof(float), n * sizeof(float), n * B, n * B, (size_t)B * sizeof(int32_t)};
+    const void *mapped[5];
+    bool in_mapped = true;
+    for (int i = 0; i < 5 && in_mapped; ++i) in_mapped = (mapped[i] = device_alias(src[i])) != nullptr;
+    if (in_mapped) {
+        if (launch_stage_inputs(mapped, dst, len, g->info.sm_count, st) != cudaSuccess) return PLACETO_ERR_CUDA;
+    } else {
+        for (int i = 0; i < 5; ++i)
+            if (cudaMemcpyAsync(dst[i], src[i], len[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+                return PLACETO_ERR_CUDA;
+    }
+    float *out_logits = static_cast<float *>(const_cast<void *>(device_alias(logits)));
+    float *out_probs = probs ? static_cast<float *>(const_cast<void *>(device_alias(probs))) : nullptr;
+    const bool out_mapped = out_logits && (!probs || out_probs) && aligned16(out_logits) &&
+                            (!probs || aligned16(out_probs));
+    if (!out_mapped) { out_logits = d_logits; out_probs = probs ? d_probs : nullptr; }
     float *X = reinterpret_cast<float *>(ws + L.X);
     float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
     float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
@@ -534,12 +561,14 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     if (s != PLACETO_OK) return s;
     s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;
-    s = run_pool(g, w, X, Hd, Hu, d_cur, B, d_logits, probs ? d_probs : nullptr, ws, L, flags, st, true);
+    s = run_pool(g, w, X, Hd, Hu, d_cur, B, out_logits, out_probs, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;
-    if (cudaMemcpyAsync(logits, d_logits, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return PLACETO_ERR_CUDA;
-    if (probs && cudaMemcpyAsync(probs, d_probs, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return PLACETO_ERR_CUDA;
+    if (!out_mapped) {
+        if (cudaMemcpyAsync(logits, d_logits, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return PLACETO_ERR_CUDA;
+        if (probs && cudaMemcpyAsync(probs, d_probs, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return PLACETO_ERR_CUDA;
+    }
     return cuda_status(cudaStreamSynchronize(st));
 }
 

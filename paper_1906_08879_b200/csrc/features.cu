@@ -4,6 +4,8 @@
 // written as X[n][B][F]. The state arrays are state-major (dev[B][n]) while X
 // is node-major, so a block transposes a 32-node x 32-state tile through
 // shared memory: loads run along nodes, stores along (state, feature).
+#include <algorithm>
+
 #include "kernels.cuh"
 
 namespace placeto {
@@ -70,7 +72,56 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
     }
 }
 
+// Gathers the host-resident inputs of one policy evaluation into device memory
+// in a single launch. The sources are page-locked host buffers that the device
+// can address; a warp reads 512 contiguous bytes per pass (16 bytes per lane), so
+// the reads cross the host link as full-size requests.
+struct StageSegments {
+    const char *src[5];
+    char *dst[5];
+    size_t bytes[5];
+};
+
+__global__ void __launch_bounds__(256)
+stage_inputs_kernel(const StageSegments s) {
+    dependents_may_start();
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const char *src = s.src[i];
+        char *dst = s.dst[i];
+        const size_t bytes = s.bytes[i];
+        size_t done = 0;
+        if (((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0) {
+            const size_t words = bytes / 16;
+            for (size_t k = tid; k < words; k += stride)
+                reinterpret_cast<uint4 *>(dst)[k] = reinterpret_cast<const uint4 *>(src)[k];
+            done = words * 16;
+        }
+        for (size_t k = done + tid; k < bytes; k += stride) dst[k] = src[k];
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_stage_inputs(const void *const (&src)[5], void *const (&dst)[5],
+                                const size_t (&bytes)[5], int sm_count, cudaStream_t stream) {
+    StageSegments s;
+    size_t total = 0;
+    for (int i = 0; i < 5; ++i) {
+        s.src[i] = static_cast<const char *>(src[i]);
+        s.dst[i] = static_cast<char *>(dst[i]);
+        s.bytes[i] = bytes[i];
+        total += bytes[i];
+    }
+    // one 16-byte word per thread up to two blocks per SM, grid-stride beyond
+    const size_t want = (total / 16 + 255) / 256 + 1;
+    const int grid = (int)std::min<size_t>(want, (size_t)2 * sm_count);
+    stage_inputs_kernel<<<grid, 256, 0, stream>>>(s);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,

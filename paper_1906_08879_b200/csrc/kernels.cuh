@@ -150,6 +150,10 @@ cudaError_t launch_features(int n, int B, int m, const float *cost, const float 
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
                             cudaStream_t stream);
 
+// Copies five host-resident, device-addressable buffers into device memory in one launch.
+cudaError_t launch_stage_inputs(const void *const (&src)[5], void *const (&dst)[5],
+                                const size_t (&bytes)[5], int sm_count, cudaStream_t stream);
+
 // episode.cu: the MDP transition between two policy evaluations of an episode
 cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream);
 cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream);

@@ -381,6 +381,38 @@ def test_policy_forward_and_host_variant_match_the_separate_calls():
     assert torch.equal(h_logits, ref["logits"].cpu()) and torch.equal(h_probs, ref["probs"].cpu())
 
 
+@pytest.mark.parametrize("pinned_in,pinned_out", [(False, False), (True, False), (False, True)])
+def test_host_variant_with_pageable_buffers(pinned_in, pinned_out):
+    """Page-locked buffers are read and written by the kernels themselves,
+    pageable ones go through copies: every mix gives the same results, also with an
+    unaligned pageable input and without the probabilities."""
+    cfg = configs.make("tiny")
+    ref = gpu_forward(cfg)
+    g, w = ref["graph"], ref["w"]
+    B, m = cfg["B"], cfg["m"]
+    ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD_HOST)
+
+    def host(a, pinned, shift=0):
+        a = np.ascontiguousarray(a)
+        if pinned:
+            return torch.from_numpy(a).pin_memory()
+        raw = np.empty(a.nbytes + 64, dtype=np.uint8)      # pageable, optionally off 16-byte alignment
+        off = (-raw.ctypes.data) % 16 + shift
+        view = raw[off:off + a.nbytes].view(a.dtype).reshape(a.shape)
+        view[...] = a
+        return torch.from_numpy(view)
+
+    ins = [host(cfg["cost"], pinned_in), host(cfg["bytes"], pinned_in), host(cfg["dev"], pinned_in, 1),
+           host(cfg["cur"], pinned_in), host(cfg["placed"], pinned_in)]
+    out = lambda: host(np.zeros((B, m), np.float32), pinned_out)
+    h_logits, h_probs = out(), out()
+    placeto.placeto_policy_forward_host(g, w, *ins, h_logits, h_probs, ws)
+    assert torch.equal(h_logits, ref["logits"].cpu()) and torch.equal(h_probs, ref["probs"].cpu())
+    only_logits = out()
+    placeto.placeto_policy_forward_host(g, w, *ins, only_logits, None, ws)
+    assert torch.equal(only_logits, ref["logits"].cpu())
+
+
 def test_two_streams_with_their_own_workspaces_do_not_interfere():
     cfg = configs.make("inception")
     ref = gpu_forward(cfg)
