@@ -65,6 +65,45 @@ __device__ __forceinline__ void fma_rows(const pair_t *w, const float *const (&i
     }
 }
 
+// ---- bulk asynchronous copies (the TMA unit moves a contiguous run of bytes from
+// global to shared memory and reports the bytes on an mbarrier) -------------------
+__device__ __forceinline__ unsigned smem_addr(const void *p) {
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, int arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect(unsigned long long *bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+// src and dst 16-byte aligned, bytes a positive multiple of 16
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes,
+                                          unsigned long long *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_addr(dst)),
+        "l"(src), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+// Waits for phase `parity` of the barrier; gives up after a bounded number of
+// polls (a copy that never lands must not hang the device) and reports it.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
+    for (int i = 0; i < (1 << 22); ++i) {
+        unsigned done;
+        asm volatile(
+            "{\n.reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(done)
+            : "r"(smem_addr(bar)), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
 template <int F4>
 __global__ void __launch_bounds__(kThreads, 1)
 pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
@@ -84,35 +123,28 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     float *hu = hd + (size_t)p.chunk_nodes * kWarps * kD;
     float *xs = hu + (size_t)p.chunk_nodes * kWarps * kD;   // [chunk][16][FP]
 
-    // ---- stage weights and the tile
-    for (int i = 0; i < 3; ++i) {
-        const float *W = a.l[i].W1;
-        for (int t = threadIdx.x; t < E * kD / 4; t += kThreads) {
-            const int k = (t * 4) / kD;
-            if (k < 2 * kD + F) __pipeline_memcpy_async(Ws + i * E * kD + t * 4, W + t * 4, 16);
-            else *reinterpret_cast<float4 *>(Ws + i * E * kD + t * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (threadIdx.x < kD) bs[i * kD + threadIdx.x] = a.l[i].b1[threadIdx.x];
+    // ---- stage weights and the tile: one bulk copy per matrix and three per node
+    // (16 states x 32 floats of H_down and H_up, 16 states x F of X are contiguous
+    // both in global and in shared memory), all reporting to one mbarrier
+    __shared__ __align__(8) unsigned long long bar;
+    const unsigned w_bytes = (unsigned)(E * kD * sizeof(float));      // F == FP here: no padding rows
+    const unsigned h_bytes = (unsigned)(nb * kD * sizeof(float)), x_bytes = (unsigned)(nb * F * sizeof(float));
+    if (threadIdx.x == 0) mbar_init(&bar, 1);
+    if (threadIdx.x < 3 * kD) bs[threadIdx.x] = a.l[threadIdx.x / kD].b1[threadIdx.x % kD];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        mbar_expect(&bar, 3 * w_bytes + (unsigned)nu * (2 * h_bytes + x_bytes));
+        for (int i = 0; i < 3; ++i) bulk_load(Ws + i * E * kD, a.l[i].W1, w_bytes, &bar);
     }
     dependency_wait();          // the embeddings may come from a kernel that is still running
-    {
-        const int per_h = nb * kD / 4;                  // 16-byte pieces per node
-        for (int t = threadIdx.x; t < nu * per_h; t += kThreads) {
-            const int q = t / per_h, off = (t - q * per_h) * 4;
-            const size_t src = ((size_t)(u0 + q) * B + b0) * kD + off;
-            __pipeline_memcpy_async(hd + (size_t)q * kWarps * kD + off, a.H[0] + src, 16);
-            __pipeline_memcpy_async(hu + (size_t)q * kWarps * kD + off, a.H[1] + src, 16);
-        }
-        const int per_x = nb * F / 4;                   // F is a multiple of 4 here, FP == F
-        for (int t = threadIdx.x; t < nu * per_x; t += kThreads) {
-            const int q = t / per_x, off = (t - q * per_x) * 4;
-            __pipeline_memcpy_async(xs + (size_t)q * kWarps * FP + off,
-                                    a.X + ((size_t)(u0 + q) * B + b0) * F + off, 16);
-        }
+    for (int t = threadIdx.x; t < 3 * nu; t += kThreads) {
+        const int q = t / 3, which = t - 3 * q;
+        const size_t row = (size_t)(u0 + q) * B + b0;
+        if (which == 0) bulk_load(hd + (size_t)q * kWarps * kD, a.H[0] + row * kD, h_bytes, &bar);
+        else if (which == 1) bulk_load(hu + (size_t)q * kWarps * kD, a.H[1] + row * kD, h_bytes, &bar);
+        else bulk_load(xs + (size_t)q * kWarps * FP, a.X + row * F, x_bytes, &bar);
     }
-    __pipeline_commit();
-    __pipeline_wait_prior(0);
-    __syncthreads();
+    const bool landed = mbar_wait(&bar, 0);
 
     if (warp >= nb) return;
     const int b = b0 + warp;
@@ -159,7 +191,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
                 }
             }
         }
-        out[i * kD + lane] = total;
+        out[i * kD + lane] = landed ? total : nanf("");   // a copy that never landed shows as NaN logits
     }
 }
 
