@@ -65,45 +65,6 @@ __device__ __forceinline__ void fma_rows(const pair_t *w, const float *const (&i
     }
 }
 
-// ---- bulk asynchronous copies (the TMA unit moves a contiguous run of bytes from
-// global to shared memory and reports the bytes on an mbarrier) -------------------
-__device__ __forceinline__ unsigned smem_addr(const void *p) {
-    return (unsigned)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, int arrivals) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect(unsigned long long *bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
-                 : "memory");
-}
-// src and dst 16-byte aligned, bytes a positive multiple of 16
-__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes,
-                                          unsigned long long *bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-            smem_addr(dst)),
-        "l"(src), "r"(bytes), "r"(smem_addr(bar))
-        : "memory");
-}
-// Waits for phase `parity` of the barrier; gives up after a bounded number of
-// polls (a copy that never lands must not hang the device) and reports it.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
-    for (int i = 0; i < (1 << 22); ++i) {
-        unsigned done;
-        asm volatile(
-            "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-            "selp.u32 %0, 1, 0, p;\n}"
-            : "=r"(done)
-            : "r"(smem_addr(bar)), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
 template <int F4>
 __global__ void __launch_bounds__(kThreads, 1)
 pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
@@ -129,13 +90,14 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     __shared__ __align__(8) unsigned long long bar;
     const unsigned w_bytes = (unsigned)(E * kD * sizeof(float));      // F == FP here: no padding rows
     const unsigned h_bytes = (unsigned)(nb * kD * sizeof(float)), x_bytes = (unsigned)(nb * F * sizeof(float));
-    if (threadIdx.x == 0) mbar_init(&bar, 1);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_expect(&bar, 3 * w_bytes + (unsigned)nu * (2 * h_bytes + x_bytes));
+    }
     if (threadIdx.x < 3 * kD) bs[threadIdx.x] = a.l[threadIdx.x / kD].b1[threadIdx.x % kD];
     __syncthreads();
-    if (threadIdx.x == 0) {
-        mbar_expect(&bar, 3 * w_bytes + (unsigned)nu * (2 * h_bytes + x_bytes));
+    if (threadIdx.x == 0)
         for (int i = 0; i < 3; ++i) bulk_load(Ws + i * E * kD, a.l[i].W1, w_bytes, &bar);
-    }
     dependency_wait();          // the embeddings may come from a kernel that is still running
     for (int t = threadIdx.x; t < 3 * nu; t += kThreads) {
         const int q = t / 3, which = t - 3 * q;

@@ -11,7 +11,7 @@
 // row from shared memory (broadcast 128-bit loads, 4 FMAs per load), combines
 // the quarters with two shuffles and adds relu(.) to the accumulator of the row's
 // set. The rows of each (state, set) are compacted into index lists while the
-// tile is staged (cp.async), so the main loop runs set by set, two rows in
+// tile is staged (bulk asynchronous copies), so the main loop runs set by set, two rows in
 // flight, without branching on the set. Warps never synchronise after staging.
 // Summation order is ascending node id per (chunk, state, set): deterministic.
 #include <cuda_pipeline.h>
@@ -102,17 +102,24 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     // per state and set: the chunk's node indices of that set, ascending  [states][3][chunk]
     uint8_t *lists = reinterpret_cast<uint8_t *>(rows + (size_t)p.chunk_nodes * kTileStates * RS);
     __shared__ int counts[kTileStates][3];
-    // ---- stage the tile: every row as one contiguous [h_down | h_up | x | 0] vector
+    // ---- stage the tile: every row as one contiguous [h_down | h_up | x | 0] vector,
+    // three bulk copies per (node, state) row reporting to one mbarrier
+    __shared__ __align__(8) unsigned long long bar;
     {
-        const int pieces = (2 * kD + F) / 4;            // 16-byte pieces per row (F multiple of 4)
-        for (int t = threadIdx.x; t < nu * nb * pieces; t += kThreads) {
-            const int r = t / pieces, k = (t - r * pieces) * 4;
+        const unsigned x_bytes = (unsigned)(F * sizeof(float)), h_bytes = (unsigned)(kD * sizeof(float));
+        if (threadIdx.x == 0) {
+            mbar_init(&bar, 1);
+            mbar_expect(&bar, (unsigned)(nu * nb) * (2 * h_bytes + x_bytes));
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < nu * nb * 3; t += kThreads) {
+            const int r = t / 3, which = t - 3 * r;
             const int q = r / nb, s = r - q * nb;
             const size_t src = (size_t)(u0 + q) * B + b0 + s;
-            const float *from = k < kD ? a.H[0] + src * kD + k
-                              : k < 2 * kD ? a.H[1] + src * kD + (k - kD)
-                                           : a.X + src * F + (k - 2 * kD);
-            __pipeline_memcpy_async(rows + ((size_t)q * kTileStates + s) * RS + k, from, 16);
+            float *dst = rows + ((size_t)q * kTileStates + s) * RS;
+            if (which == 0) bulk_load(dst, a.H[0] + src * kD, h_bytes, &bar);
+            else if (which == 1) bulk_load(dst + kD, a.H[1] + src * kD, h_bytes, &bar);
+            else bulk_load(dst + 2 * kD, a.X + src * F, x_bytes, &bar);
         }
         const int pad = RS - (2 * kD + F);
         for (int t = threadIdx.x; t < nu * nb * pad; t += kThreads) {
@@ -151,9 +158,8 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
         w2[k] = in_range ? a.l[2].W1[kk * kD + col] : 0.f;
     }
     const float bias0 = a.l[0].b1[col], bias1 = a.l[1].b1[col], bias2 = a.l[2].b1[col];
-    __pipeline_commit();
-    __pipeline_wait_prior(0);
-    __syncthreads();
+    const bool landed = mbar_wait(&bar, 0);
+    __syncthreads();            // lists, counts and the zero padding written by other threads
 
     for (int s = 0; s < nb; ++s) {
         const float *rows_s = rows + (size_t)s * RS + quarter * KQ;
@@ -163,9 +169,10 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
         const float acc2 = set_sum<KQ, RS>(w2, bias2, ls + 2 * p.chunk_nodes, counts[s][2], rows_s);
         if (quarter == 0) {
             float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + col;
-            out[0] = acc0;
-            out[kD] = acc1;
-            out[2 * kD] = acc2;
+            // a copy that never landed shows as NaN logits
+            out[0] = landed ? acc0 : nanf("");
+            out[kD] = landed ? acc1 : nanf("");
+            out[2 * kD] = landed ? acc2 : nanf("");
         }
     }
 }
