@@ -557,7 +557,10 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     float *X = reinterpret_cast<float *>(ws + L.X);
     float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
     float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
-    s = cuda_status(launch_features(g->host.n, B, w->m, d_cost, d_bytes, d_dev, d_cur, d_placed, X, st));
+    // after the gather kernel the whole chain overlaps: the set-up of the message
+    // passing kernel (weights, schedule) runs while the inputs cross the host link
+    s = cuda_status(launch_features(g->host.n, B, w->m, d_cost, d_bytes, d_dev, d_cur, d_placed, X, st,
+                                    in_mapped));
     if (s != PLACETO_OK) return s;
     s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
     if (s != PLACETO_OK) return s;

@@ -26,6 +26,7 @@ features_kernel(int n, int B, int m, const float *__restrict__ cost,
     __shared__ float s_cost[kTile], s_bytes[kTile];
     const int v0 = blockIdx.x * kTile, b0 = blockIdx.y * kTile;
     const int F = m + 4;
+    dependency_wait();          // the inputs may come from the gather kernel of the same call
     for (int i = threadIdx.x; i < kTile * kTile; i += blockDim.x) {
         const int bl = i / kTile, vl = i % kTile;
         const int b = b0 + bl, v = v0 + vl;
@@ -125,11 +126,12 @@ cudaError_t launch_stage_inputs(const void *const (&src)[5], void *const (&dst)[
 
 cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, bool overlap) {
     dim3 grid((n + kTile - 1) / kTile, (B + kTile - 1) / kTile);
-    features_kernel<<<grid, 256, 0, stream>>>(n, B, m, cost, bytes, dev, cur, placed, X);
+    cudaError_t err = launch_overlapped(overlap, features_kernel, grid, dim3(256), 0, stream, n, B, m, cost,
+                                        bytes, dev, cur, placed, X);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace placeto

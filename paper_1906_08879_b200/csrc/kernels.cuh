@@ -190,7 +190,7 @@ cudaError_t launch_overlapped(bool overlap, void (*kern)(KArgs...), dim3 grid, d
 // features.cu
 cudaError_t launch_features(int n, int B, int m, const float *cost, const float *bytes,
                             const uint8_t *dev, const int *cur, const uint8_t *placed, float *X,
-                            cudaStream_t stream);
+                            cudaStream_t stream, bool overlap = false);
 
 // Copies five host-resident, device-addressable buffers into device memory in one launch.
 cudaError_t launch_stage_inputs(const void *const (&src)[5], void *const (&dst)[5],
