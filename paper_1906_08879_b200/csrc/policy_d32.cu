@@ -5,14 +5,13 @@
 // sums that the head kernel adds up in chunk order.
 //
 // A block first copies its whole tile (chunk x 16 states of H_down, H_up, X) and
-// the three weight matrices into shared memory with cp.async. Warp w owns state
+// the three weight matrices into shared memory with bulk asynchronous copies
+// (one per matrix, three per node, counted on an mbarrier). Warp w owns state
 // w of the tile. For each set i in turn it loads column `lane` of W_i into
 // registers, scans the relation row of its state's current node over the chunk
 // (ballot), and pushes the rows of set i through the 32 x (64 + F) product two at
 // a time, reading the inputs as broadcast 128-bit shared loads; the sums stay in
 // registers. Summation order is ascending node id: deterministic.
-#include <cuda_pipeline.h>
-
 #include <algorithm>
 
 #include "kernels.cuh"

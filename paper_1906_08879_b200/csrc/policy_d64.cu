@@ -14,8 +14,6 @@
 // tile is staged (bulk asynchronous copies), so the main loop runs set by set, two rows in
 // flight, without branching on the set. Warps never synchronise after staging.
 // Summation order is ascending node id per (chunk, state, set): deterministic.
-#include <cuda_pipeline.h>
-
 #include <algorithm>
 
 #include "kernels.cuh"
