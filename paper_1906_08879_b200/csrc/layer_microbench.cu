@@ -239,6 +239,45 @@ __global__ void k_layer_split(float *out, unsigned *t, const float *wsrc) {
     if (threadIdx.x == 0) t[0] = t1 - t0;
 }
 
+// Throughput of 128-bit shared loads by address pattern: eight warps each issue
+// kIters x 16 loads whose 16-byte chunks are spread over the lanes as `pattern`
+// says (no bank conflicts in any of them); reports cycles per load per SM. The
+// loads are volatile so that none is merged or hoisted.
+__global__ void __launch_bounds__(256) k_lds_pattern(float *out, unsigned *t, int pattern) {
+    __shared__ __align__(16) float buf[8192];
+    for (int i = threadIdx.x; i < 8192; i += blockDim.x) buf[i] = (float)i;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int off;   // float offset of this lane's chunk
+    switch (pattern) {
+        case 0: off = 0; break;                    // one address for the warp
+        case 1: off = (lane >> 4) * 36; break;     // one per half-warp
+        case 2: off = (lane >> 3) * 36; break;     // one per quarter-warp (8 consecutive lanes)
+        case 3: off = (lane >> 2) * 76; break;     // one per group of 4 lanes: 2 per quarter-warp
+        case 4: off = (lane & 1) * 36; break;      // 2 addresses alternating by lane
+        case 5: off = (lane & 3) * 36; break;      // 4 addresses by lane mod 4: 4 per quarter-warp
+        case 6: off = (lane & 7) * 4; break;       // 8 adjacent chunks, the same in every quarter-warp
+        default: off = lane * 4; break;            // 32 distinct adjacent chunks
+    }
+    const unsigned base = (unsigned)__cvta_generic_to_shared(buf + off + warp * 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    const unsigned t0 = clk();
+    for (int it = 0; it < kIters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            float4 v;
+            asm volatile("ld.volatile.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                         : "r"(base + (unsigned)(u % 8) * 256u));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+    }
+    const unsigned t1 = clk();
+    __syncthreads();
+    if (threadIdx.x == 0) *t = t1 - t0;
+    out[threadIdx.x] = acc.x + acc.y + acc.z + acc.w;
+}
+
 int main() {
     float *out, *w;
     unsigned *t, h = 0;
@@ -286,6 +325,19 @@ int main() {
     LAYER("packed fma (f32x2)", (k_layer_packed<2>), 2)
     LAYER("half-warp split", (k_layer_split<2>), 2)
     LAYER("fma, 2 accumulators", (k_layer<4, 2>), 4)
+    const char *patterns[] = {"one address per warp", "one per half-warp", "one per quarter-warp",
+                              "one per 4 lanes (2 per quarter-warp)", "2 alternating by lane",
+                              "4 by lane mod 4 (4 per quarter-warp)", "8 adjacent chunks per quarter-warp",
+                              "32 distinct chunks"};
+    for (int pat = 0; pat < 8; ++pat) {
+        for (int rep = 0; rep < 2; ++rep) {
+            k_lds_pattern<<<1, 256>>>(out, t, pat);
+            cudaDeviceSynchronize();
+            cudaMemcpy(&h, t, 4, cudaMemcpyDeviceToHost);
+        }
+        printf("128-bit shared load, %-38s %5.2f cycles per load per SM, 8 warps  (%s)\n", patterns[pat],
+               h / (double)kIters / (16 * 8), cudaGetErrorString(cudaGetLastError()));
+    }
     cudaFree(out); cudaFree(t); cudaFree(w);
     return 0;
 }
