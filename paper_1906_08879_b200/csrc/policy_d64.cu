@@ -3,15 +3,16 @@
 //   l_i(e_u),   e_u = [h_down_u || h_up_u || x_u],   i = set of u relative to cur[b],
 // for a tile of states per block, in the layout the head kernel adds up.
 //
-// The three 140 x 64 matrices (with F = 12) are too large to switch per set, so
-// they stay resident, split over the block: eight warps, warp w owns output
-// columns [8w, 8w + 8), lane (quarter, col) keeps one quarter of the inner
-// dimension of its column for all three sets (3 x 36 registers). Every warp
-// walks all rows (state, node) of the block's tile: it reads its quarter of the
-// row from shared memory (broadcast 128-bit loads, 4 FMAs per load), combines
-// the quarters with two shuffles and adds relu(.) to the accumulator of the row's
-// set. The rows of each (state, set) are compacted into index lists while the
-// tile is staged (bulk asynchronous copies), so the main loop runs set by set, two rows in
+// The block works one set at a time: lane (quarter, pair) keeps two adjacent
+// columns of W_i for one quarter of the inner dimension (2 x 36 registers), four
+// warps cover the 64 columns, and the two groups of four warps take alternate
+// states of the tile. A warp reads its quarter of a row from shared memory (one
+// address per quarter-warp, the cheapest pattern of a 128-bit load, feeding 8
+// FMAs per lane), combines the quarters with two shuffles per column and adds
+// relu(.) to the sum of the (state, set) list it is walking. A row is read by
+// four warps instead of the eight that one column per lane needs. The rows of
+// each (state, set) are compacted into index lists while the tile is staged
+// (bulk asynchronous copies), so the main loop runs list by list, two rows in
 // flight, without branching on the set. Warps never synchronise after staging.
 // Summation order is ascending node id per (chunk, state, set): deterministic.
 #include <algorithm>
@@ -32,50 +33,51 @@ struct Pool64Plan {
     size_t smem_bytes;
 };
 
-// Sum over one set's rows (node indices in `list`) of relu(bias + row . w), this
-// lane's column; two rows in flight, four accumulators each.
+// Sum over one set's rows (node indices in `list`) of relu(bias + row . w) for this
+// lane's two columns; two rows in flight, four accumulators per row and column.
 template <int KQ, int RS>
-__device__ __forceinline__ float set_sum(const float (&w)[KQ], float bias, const uint8_t *list,
-                                         int count, const float *rows_s) {
-    float total = 0.f;
-    int i = 0;
-    for (; i + 2 <= count; i += 2) {
+__device__ __forceinline__ float2 set_sum(const float (&w)[2][KQ], float2 bias, const uint8_t *list,
+                                          int count, const float *rows_s) {
+    float2 total = make_float2(0.f, 0.f);
+    for (int i = 0; i < count; i += 2) {
+        const bool two = i + 1 < count;
         const float *in0 = rows_s + (size_t)list[i] * (kTileStates * RS);
-        const float *in1 = rows_s + (size_t)list[i + 1] * (kTileStates * RS);
-        float a[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        const float *in1 = rows_s + (size_t)list[two ? i + 1 : i] * (kTileStates * RS);
+        float a[2][2][4];
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) a[r][c][q] = 0.f;
 #pragma unroll
         for (int k = 0; k < KQ; k += 4) {
             const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
             const float4 v = *reinterpret_cast<const float4 *>(in1 + k);
-            a[0][0] = fmaf(u.x, w[k], a[0][0]);     a[1][0] = fmaf(v.x, w[k], a[1][0]);
-            a[0][1] = fmaf(u.y, w[k + 1], a[0][1]); a[1][1] = fmaf(v.y, w[k + 1], a[1][1]);
-            a[0][2] = fmaf(u.z, w[k + 2], a[0][2]); a[1][2] = fmaf(v.z, w[k + 2], a[1][2]);
-            a[0][3] = fmaf(u.w, w[k + 3], a[0][3]); a[1][3] = fmaf(v.w, w[k + 3], a[1][3]);
-        }
-        float s0 = (a[0][0] + a[0][1]) + (a[0][2] + a[0][3]);
-        float s1 = (a[1][0] + a[1][1]) + (a[1][2] + a[1][3]);
-        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);
-        s1 += __shfl_xor_sync(0xffffffffu, s1, 8);
-        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
-        s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
-        total += fmaxf(s0 + bias, 0.f);
-        total += fmaxf(s1 + bias, 0.f);
-    }
-    if (i < count) {
-        const float *in0 = rows_s + (size_t)list[i] * (kTileStates * RS);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-        for (int k = 0; k < KQ; k += 4) {
-            const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
-            a0 = fmaf(u.x, w[k], a0);
-            a1 = fmaf(u.y, w[k + 1], a1);
-            a2 = fmaf(u.z, w[k + 2], a2);
-            a3 = fmaf(u.w, w[k + 3], a3);
+            for (int c = 0; c < 2; ++c) {
+                a[0][c][0] = fmaf(u.x, w[c][k], a[0][c][0]);     a[1][c][0] = fmaf(v.x, w[c][k], a[1][c][0]);
+                a[0][c][1] = fmaf(u.y, w[c][k + 1], a[0][c][1]); a[1][c][1] = fmaf(v.y, w[c][k + 1], a[1][c][1]);
+                a[0][c][2] = fmaf(u.z, w[c][k + 2], a[0][c][2]); a[1][c][2] = fmaf(v.z, w[c][k + 2], a[1][c][2]);
+                a[0][c][3] = fmaf(u.w, w[c][k + 3], a[0][c][3]); a[1][c][3] = fmaf(v.w, w[c][k + 3], a[1][c][3]);
+            }
         }
-        float s0 = (a0 + a1) + (a2 + a3);
-        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);
-        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
-        total += fmaxf(s0 + bias, 0.f);
+        float sum[2][2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                float t = (a[r][c][0] + a[r][c][1]) + (a[r][c][2] + a[r][c][3]);
+                t += __shfl_xor_sync(0xffffffffu, t, 8);       // the four quarters of the inner dimension
+                t += __shfl_xor_sync(0xffffffffu, t, 16);
+                sum[r][c] = t;
+            }
+        total.x += fmaxf(sum[0][0] + bias.x, 0.f);
+        total.y += fmaxf(sum[0][1] + bias.y, 0.f);
+        if (two) {
+            total.x += fmaxf(sum[1][0] + bias.x, 0.f);
+            total.y += fmaxf(sum[1][1] + bias.y, 0.f);
+        }
     }
     return total;
 }
@@ -90,7 +92,9 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     dependents_may_start();
     dependency_wait();          // the embeddings may come from a kernel that is still running
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int quarter = lane >> 3, col = warp * 8 + (lane & 7);
+    // warps 0-3 and 4-7 each cover all 64 columns (16 per warp, two per lane) and share the
+    // tile's states between them; lane (quarter, pair) keeps a quarter of the inner dimension
+    const int quarter = lane >> 3, col = (warp & 3) * 16 + 2 * (lane & 7), group = warp >> 2;
     const int n = a.n, B = a.B, F = a.F;
     const int chunk = blockIdx.x;
     const int u0 = chunk * p.chunk_nodes, nu = min(n, u0 + p.chunk_nodes) - u0;
@@ -145,33 +149,35 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
         }
         if (lane < 3) counts[warp][lane] = lane == 0 ? cnt[0] : (lane == 1 ? cnt[1] : cnt[2]);
     }
-    // ---- this lane's weights: column `col`, its quarter of the inner dimension, three sets
-    float w0[KQ], w1[KQ], w2[KQ];
+    // ---- one set at a time: this lane's two columns of W_i, its quarter of the inner dimension
+    float w[2][KQ];
+    auto load_set = [&](int i) {
 #pragma unroll
-    for (int k = 0; k < KQ; ++k) {
-        const int kk = quarter * KQ + k;
-        const bool in_range = kk < 2 * kD + F;
-        w0[k] = in_range ? a.l[0].W1[kk * kD + col] : 0.f;
-        w1[k] = in_range ? a.l[1].W1[kk * kD + col] : 0.f;
-        w2[k] = in_range ? a.l[2].W1[kk * kD + col] : 0.f;
-    }
-    const float bias0 = a.l[0].b1[col], bias1 = a.l[1].b1[col], bias2 = a.l[2].b1[col];
+        for (int k = 0; k < KQ; ++k) {
+            const int kk = quarter * KQ + k;
+            const float2 v = kk < 2 * kD + F ? *reinterpret_cast<const float2 *>(a.l[i].W1 + kk * kD + col)
+                                             : make_float2(0.f, 0.f);
+            w[0][k] = v.x;
+            w[1][k] = v.y;
+        }
+    };
+    load_set(0);
     const bool landed = mbar_wait(&bar, 0);
     __syncthreads();            // lists, counts and the zero padding written by other threads
 
-    for (int s = 0; s < nb; ++s) {
-        const float *rows_s = rows + (size_t)s * RS + quarter * KQ;
-        const uint8_t *ls = lists + (size_t)s * 3 * p.chunk_nodes;
-        const float acc0 = set_sum<KQ, RS>(w0, bias0, ls, counts[s][0], rows_s);
-        const float acc1 = set_sum<KQ, RS>(w1, bias1, ls + p.chunk_nodes, counts[s][1], rows_s);
-        const float acc2 = set_sum<KQ, RS>(w2, bias2, ls + 2 * p.chunk_nodes, counts[s][2], rows_s);
-        if (quarter == 0) {
-            float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + col;
-            // a copy that never landed shows as NaN logits
-            out[0] = landed ? acc0 : nanf("");
-            out[kD] = landed ? acc1 : nanf("");
-            out[2 * kD] = landed ? acc2 : nanf("");
+    for (int i = 0; i < 3; ++i) {
+        const float2 bias = *reinterpret_cast<const float2 *>(a.l[i].b1 + col);
+        for (int s = group; s < nb; s += 2) {
+            const float *rows_s = rows + (size_t)s * RS + quarter * KQ;
+            const uint8_t *ls = lists + ((size_t)s * 3 + i) * p.chunk_nodes;
+            const float2 acc = set_sum<KQ, RS>(w, bias, ls, counts[s][i], rows_s);
+            if (quarter == 0) {
+                // a copy that never landed shows as NaN logits
+                float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + i * kD + col;
+                *reinterpret_cast<float2 *>(out) = landed ? acc : make_float2(nanf(""), nanf(""));
+            }
         }
+        if (i < 2) load_set(i + 1);
     }
 }
 
