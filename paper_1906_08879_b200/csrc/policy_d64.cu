@@ -33,53 +33,48 @@ struct Pool64Plan {
     size_t smem_bytes;
 };
 
+constexpr int kCols = 4;      // adjacent output columns per lane
+
 // Sum over one set's rows (node indices in `list`) of relu(bias + row . w) for this
-// lane's two columns; two rows in flight, four accumulators per row and column.
+// lane's columns; two rows in flight, two accumulators per row and column.
 template <int KQ, int RS>
-__device__ __forceinline__ float2 set_sum(const float (&w)[2][KQ], float2 bias, const uint8_t *list,
-                                          int count, const float *rows_s) {
-    float2 total = make_float2(0.f, 0.f);
+__device__ __forceinline__ void set_sum(const float (&w)[kCols][KQ], const float (&bias)[kCols],
+                                        const uint8_t *list, int count, const float *rows_s,
+                                        float (&total)[kCols]) {
+#pragma unroll
+    for (int c = 0; c < kCols; ++c) total[c] = 0.f;
     for (int i = 0; i < count; i += 2) {
         const bool two = i + 1 < count;
         const float *in0 = rows_s + (size_t)list[i] * (kTileStates * RS);
         const float *in1 = rows_s + (size_t)list[two ? i + 1 : i] * (kTileStates * RS);
-        float a[2][2][4];
+        float a[2][kCols][2];
 #pragma unroll
         for (int r = 0; r < 2; ++r)
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) a[r][c][q] = 0.f;
+            for (int c = 0; c < kCols; ++c) a[r][c][0] = a[r][c][1] = 0.f;
 #pragma unroll
         for (int k = 0; k < KQ; k += 4) {
             const float4 u = *reinterpret_cast<const float4 *>(in0 + k);
             const float4 v = *reinterpret_cast<const float4 *>(in1 + k);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < kCols; ++c) {
                 a[0][c][0] = fmaf(u.x, w[c][k], a[0][c][0]);     a[1][c][0] = fmaf(v.x, w[c][k], a[1][c][0]);
                 a[0][c][1] = fmaf(u.y, w[c][k + 1], a[0][c][1]); a[1][c][1] = fmaf(v.y, w[c][k + 1], a[1][c][1]);
-                a[0][c][2] = fmaf(u.z, w[c][k + 2], a[0][c][2]); a[1][c][2] = fmaf(v.z, w[c][k + 2], a[1][c][2]);
-                a[0][c][3] = fmaf(u.w, w[c][k + 3], a[0][c][3]); a[1][c][3] = fmaf(v.w, w[c][k + 3], a[1][c][3]);
+                a[0][c][0] = fmaf(u.z, w[c][k + 2], a[0][c][0]); a[1][c][0] = fmaf(v.z, w[c][k + 2], a[1][c][0]);
+                a[0][c][1] = fmaf(u.w, w[c][k + 3], a[0][c][1]); a[1][c][1] = fmaf(v.w, w[c][k + 3], a[1][c][1]);
             }
         }
-        float sum[2][2];
 #pragma unroll
-        for (int r = 0; r < 2; ++r)
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                float t = (a[r][c][0] + a[r][c][1]) + (a[r][c][2] + a[r][c][3]);
-                t += __shfl_xor_sync(0xffffffffu, t, 8);       // the four quarters of the inner dimension
-                t += __shfl_xor_sync(0xffffffffu, t, 16);
-                sum[r][c] = t;
-            }
-        total.x += fmaxf(sum[0][0] + bias.x, 0.f);
-        total.y += fmaxf(sum[0][1] + bias.y, 0.f);
-        if (two) {
-            total.x += fmaxf(sum[1][0] + bias.x, 0.f);
-            total.y += fmaxf(sum[1][1] + bias.y, 0.f);
+        for (int c = 0; c < kCols; ++c) {
+            float t0 = a[0][c][0] + a[0][c][1], t1 = a[1][c][0] + a[1][c][1];
+            t0 += __shfl_xor_sync(0xffffffffu, t0, 8);         // the four quarters of the inner dimension
+            t1 += __shfl_xor_sync(0xffffffffu, t1, 8);
+            t0 += __shfl_xor_sync(0xffffffffu, t0, 16);
+            t1 += __shfl_xor_sync(0xffffffffu, t1, 16);
+            total[c] += fmaxf(t0 + bias[c], 0.f);
+            if (two) total[c] += fmaxf(t1 + bias[c], 0.f);
         }
     }
-    return total;
 }
 
 template <int F4>
@@ -92,9 +87,10 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     dependents_may_start();
     dependency_wait();          // the embeddings may come from a kernel that is still running
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // warps 0-3 and 4-7 each cover all 64 columns (16 per warp, two per lane) and share the
-    // tile's states between them; lane (quarter, pair) keeps a quarter of the inner dimension
-    const int quarter = lane >> 3, col = (warp & 3) * 16 + 2 * (lane & 7), group = warp >> 2;
+    // four groups of two warps each cover all 64 columns (32 per warp, four per lane) and share
+    // the tile's states between them; a lane keeps a quarter of the inner dimension
+    constexpr int kGroups = kWarps / 2;
+    const int quarter = lane >> 3, col = (warp & 1) * 32 + kCols * (lane & 7), group = warp >> 1;
     const int n = a.n, B = a.B, F = a.F;
     const int chunk = blockIdx.x;
     const int u0 = chunk * p.chunk_nodes, nu = min(n, u0 + p.chunk_nodes) - u0;
@@ -149,16 +145,15 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
         }
         if (lane < 3) counts[warp][lane] = lane == 0 ? cnt[0] : (lane == 1 ? cnt[1] : cnt[2]);
     }
-    // ---- one set at a time: this lane's two columns of W_i, its quarter of the inner dimension
-    float w[2][KQ];
+    // ---- one set at a time: this lane's four columns of W_i, its quarter of the inner dimension
+    float w[kCols][KQ];
     auto load_set = [&](int i) {
 #pragma unroll
         for (int k = 0; k < KQ; ++k) {
             const int kk = quarter * KQ + k;
-            const float2 v = kk < 2 * kD + F ? *reinterpret_cast<const float2 *>(a.l[i].W1 + kk * kD + col)
-                                             : make_float2(0.f, 0.f);
-            w[0][k] = v.x;
-            w[1][k] = v.y;
+            const float4 v = kk < 2 * kD + F ? *reinterpret_cast<const float4 *>(a.l[i].W1 + kk * kD + col)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            w[0][k] = v.x; w[1][k] = v.y; w[2][k] = v.z; w[3][k] = v.w;
         }
     };
     load_set(0);
@@ -166,15 +161,19 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     __syncthreads();            // lists, counts and the zero padding written by other threads
 
     for (int i = 0; i < 3; ++i) {
-        const float2 bias = *reinterpret_cast<const float2 *>(a.l[i].b1 + col);
-        for (int s = group; s < nb; s += 2) {
+        const float4 b4 = *reinterpret_cast<const float4 *>(a.l[i].b1 + col);
+        const float bias[kCols] = {b4.x, b4.y, b4.z, b4.w};
+        for (int s = group; s < nb; s += kGroups) {
             const float *rows_s = rows + (size_t)s * RS + quarter * KQ;
             const uint8_t *ls = lists + ((size_t)s * 3 + i) * p.chunk_nodes;
-            const float2 acc = set_sum<KQ, RS>(w, bias, ls, counts[s][i], rows_s);
+            float acc[kCols];
+            set_sum<KQ, RS>(w, bias, ls, counts[s][i], rows_s, acc);
             if (quarter == 0) {
                 // a copy that never landed shows as NaN logits
                 float *out = a.partial + ((size_t)chunk * B + b0 + s) * 3 * kD + i * kD + col;
-                *reinterpret_cast<float2 *>(out) = landed ? acc : make_float2(nanf(""), nanf(""));
+                const float bad = nanf("");
+                *reinterpret_cast<float4 *>(out) = landed ? make_float4(acc[0], acc[1], acc[2], acc[3])
+                                                          : make_float4(bad, bad, bad, bad);
             }
         }
         if (i < 2) load_set(i + 1);
