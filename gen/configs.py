@@ -15,9 +15,11 @@ _CONFIGS = {
     "inception": (graphs.inception_shaped, 2, 4, 32, 256),
     "nmt": (graphs.nmt_shaped, 3, 4, 32, 256),
     "nasnet": (graphs.nasnet_shaped, 4, 8, 64, 512),
+    # same recipe with the shorter op chains and two lanes per op (half the depth): timed beside "nasnet"
+    "nasnet_wide": (graphs.nasnet_shaped_wide, 4, 8, 64, 512),
 }
 
-NAMES = tuple(_CONFIGS) + ("sweep",)
+NAMES = ("tiny", "inception", "nmt", "nasnet", "sweep")
 
 
 def _pack(name, n, src, dst, m, d, cost, nbytes, dev, cur, placed, weights):

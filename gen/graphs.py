@@ -154,38 +154,55 @@ def nmt_shaped(seed: int = 3, steps: int = 40, enc_layers: int = 2,
 
 
 _NAS_OPS = (1, 3, 16, 16, 16, 4)   # identity, pool, sep-conv 3/5/7, 1x1 conv
+_NAS_OPS_SHORT = (1, 2, 8, 8, 8, 3)
 
 
-def nasnet_shaped(seed: int = 4, cells: int = 18, blocks: int = 5):
+def nasnet_shaped(seed: int = 4, cells: int = 18, blocks: int = 5, ops=_NAS_OPS, adapter: int = 4,
+                  lanes: int = 1):
     """A stack of NAS cells.
 
     A cell adapts the outputs of the two preceding cells through 1x1 adapter
-    chains (4 nodes each). Each of its blocks picks two inputs uniformly among
-    the adapted inputs and the outputs of earlier blocks of the cell, passes
-    each through an op drawn uniformly from {identity: 1 node, pool: 3,
-    separable conv with kernel 3/5/7: a chain of 16, 1x1 conv: 4} and adds
-    them. Block outputs nobody used are joined by the cell's concat node.
+    chains (`adapter` nodes each). Each of its blocks picks two inputs uniformly
+    among the adapted inputs and the outputs of earlier blocks of the cell, passes
+    each through an op drawn uniformly from {identity: 1 node, pool, separable
+    conv with kernel 3/5/7, 1x1 conv} (chain lengths in `ops`) and adds them.
+    Block outputs nobody used are joined by the cell's concat node. With
+    `lanes` > 1 every op but the identity runs as that many parallel chains
+    (a grouped execution of the op) that meet in the block's add node.
+
+    The default (chains of 3 / 16 / 4, one lane) reaches the ~2000 nodes of the
+    configuration by lengthening the chains: depth 744. `nasnet_shaped_wide`
+    keeps chains of 2 / 8 / 3 and reaches the same size with two lanes per op:
+    half the depth, twice the level width.
     """
     rng = _rng(seed)
     b = _Builder()
     prev2 = b.node()
     prev1 = b.node(prev2)
     for _ in range(cells):
-        hidden = [b.chain(prev1, 4), b.chain(prev2, 4)]
+        hidden = [b.chain(prev1, adapter), b.chain(prev2, adapter)]
         used = [False, False]
         for _ in range(blocks):
             ends = []
             for _ in range(2):
                 pick = int(rng.integers(0, len(hidden)))
                 used[pick] = True
-                op = _NAS_OPS[int(rng.integers(0, len(_NAS_OPS)))]
-                ends.append(b.chain(hidden[pick], op))
+                op = ops[int(rng.integers(0, len(ops)))]
+                for _ in range(1 if op == 1 else lanes):
+                    ends.append(b.chain(hidden[pick], op))
             hidden.append(b.node(*ends))
             used.append(False)
         loose = [h for h, u in zip(hidden[2:], used[2:]) if not u]
         out = b.node(*loose)
         prev2, prev1 = prev1, out
     return b.done()
+
+
+def nasnet_shaped_wide(seed: int = 4):
+    """The NAS-cell stack with the shorter op chains (pool 2, separable conv 8,
+    1x1 conv 3, adapters 3) and two lanes per op: about the same node count as
+    `nasnet_shaped`, half its depth."""
+    return nasnet_shaped(seed, ops=_NAS_OPS_SHORT, adapter=3, lanes=2)
 
 
 def enas_conv_shaped(seed: int, target_n: int):

@@ -14,7 +14,9 @@
  *
  * Conventions
  *   - Pointers are marked HOST or DEVICE. All DEVICE pointers must be 16-byte
- *     aligned and belong to the device that was current at placeto_graph_create.
+ *     aligned and belong to the device that was current at placeto_graph_create;
+ *     that device must be current again at every call (PLACETO_ERR_INVALID_ARG
+ *     otherwise).
  *   - The caller owns every buffer (inputs, outputs, weights, workspace); the
  *     library owns only placeto_graph objects. Forward calls allocate nothing,
  *     do not synchronise (except the _host variant, see there) and run
@@ -50,8 +52,10 @@ typedef enum {
     PLACETO_ERR_UNSUPPORTED = 4, /* dimensions beyond the limits below, or flag not applicable */
     PLACETO_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
     PLACETO_ERR_NO_MEMORY = 6,   /* host or device allocation failed in graph_create */
-    PLACETO_ERR_SCRATCH_LIMIT = 7 /* batch too large for the built-in scratch of
+    PLACETO_ERR_SCRATCH_LIMIT = 7,/* batch too large for the built-in scratch of
                                      placeto_policy_logits_static */
+    PLACETO_ERR_TIMEOUT = 8      /* a bounded wait inside a kernel ran out (reported through the
+                                     status word, see placeto_last_status) */
 } placeto_status;
 
 /* Limits of the library. */
@@ -161,6 +165,9 @@ typedef struct {
                                   d = 64 otherwise takes */
 #define PLACETO_TENSOR 32u     /* use the tensor-core kernel of step 2 wherever it applies
                                   (d = 32 or 64), also where the library would pick the FMA one */
+#define PLACETO_TCGEN05 64u    /* d = 64: take the kernel built on tcgen05.mma with accumulators in tensor
+                                  memory instead of the warp-level (mma.sync) tensor-core kernel that is
+                                  the default there (measured slower at the configured batch sizes) */
 
 typedef enum {
     PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */
@@ -296,7 +303,7 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
 
 /*
  * Simulated run time of P placements of the graph under the event-based execution
- * model of the paper's simulator (Appendix A.4): one operation at a time per
+ * model of the paper's simulator (Appendix A.5): one operation at a time per
  * device, taken from a FIFO queue of runnable operations; one output tensor at a
  * time per device bus, overlapping with compute; an operation becomes runnable when
  * all parents have finished and their outputs have arrived on its device; an
@@ -322,7 +329,7 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
 /*
  * Gradient of the training objective with respect to every weight and bias of the
  * policy, for a batch of B states (Appendix A.1 of the paper: REINFORCE,
- * sum_b grad log pi(a_b | s_b) * A_b with A_b = return minus baseline; Appendix A.6:
+ * sum_b grad log pi(a_b | s_b) * A_b with A_b = return minus baseline; Appendix A.7:
  * an entropy term that encourages exploration):
  *     J = sum_b advantages[b] * log pi(actions[b] | s_b) + beta * sum_b H(pi(. | s_b)),
  *     H(p) = - sum_k p_k log p_k.
@@ -385,6 +392,34 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
                                             const float *H_up, const int32_t *cur, int32_t B,
                                             float *logits, float *probs, uint32_t flags,
                                             void *stream);
+
+/*
+ * What the kernels of the most recent call on `g` reported, read back after `stream` has
+ * drained (this call synchronises it). The library's kernels never wait without a limit: a
+ * wait on an asynchronous copy or on another warp that runs out makes the kernel leave, turn
+ * the affected outputs into NaN and write a 16-byte record into the first bytes of the call's
+ * workspace (the first 256 bytes of every workspace are reserved for it); a library built with
+ * -DPLACETO_DEBUG also records indices that its kernels found out of range (reported as
+ * PLACETO_ERR_INVALID_ARG; those accesses are skipped, nothing traps). The record carries the
+ * number of the call that wrote it, so nothing has to be cleared between calls and the
+ * contents of a fresh workspace cannot be mistaken for a report.
+ *   workspace : the workspace of that call, or NULL after placeto_policy_logits_static
+ *               (its record sits at the start of the built-in scratch).
+ * Returns PLACETO_OK, PLACETO_ERR_TIMEOUT, PLACETO_ERR_INVALID_ARG (debug build) or
+ * PLACETO_ERR_CUDA (the read itself failed). Calls on one graph object from several host
+ * threads share the call counter: ask before the next call is issued.
+ */
+placeto_status placeto_last_status(const placeto_graph *g, const void *workspace, void *stream);
+
+/*
+ * Runs the time-out path on purpose, for tests of the error channel (the paper has no
+ * counterpart): one tiny kernel announces more bytes to a barrier than its copy delivers,
+ * polls a few thousand times and gives up exactly as the library's kernels would, reporting
+ * PLACETO_ERR_TIMEOUT to placeto_last_status. Nothing faults, traps or hangs; the device stays
+ * usable. workspace: DEVICE, at least 256 bytes.
+ */
+placeto_status placeto_debug_wait_timeout(const placeto_graph *g, void *workspace, size_t workspace_bytes,
+                                          void *stream);
 
 /* Number of kernels the most recent forward call of this thread launched (for accounting). */
 int32_t placeto_last_launch_count(void);

@@ -2,7 +2,7 @@
 
 Appendix A.1 of the Placeto paper updates the parameters with
     sum_i grad_theta log pi(a_i | s_i) * (return_i - baseline_i)
-(REINFORCE with a baseline), and Appendix A.6 adds an entropy term to the loss
+(REINFORCE with a baseline), and Appendix A.7 adds an entropy term to the loss
 to encourage exploration. For a batch of B states with their chosen actions
 a_b, advantages A_b (return minus baseline, an input here) and an entropy
 factor beta, this module returns the gradient, with respect to every weight

@@ -1,5 +1,5 @@
 """CPU checker of the placement runtime simulator (test infrastructure only):
-the event-based execution model of Appendix A.4 ("Simulator") of the Placeto
+the event-based execution model of Appendix A.5 ("Simulator") of the Placeto
 paper, written out plainly with a priority queue of events.
 
 Model (paper): every device d has a FIFO queue of runnable operations and runs

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libplaceto.so")
 
 # flags and enums of placeto.h
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
-PLACETO_FMA_ONLY, PLACETO_TENSOR = 16, 32
+PLACETO_FMA_ONLY, PLACETO_TENSOR, PLACETO_TCGEN05 = 16, 32, 64
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
 CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE, CALL_EMBED_ROUNDS, CALL_GRADIENT = 0, 1, 2, 3, 4, 5, 6
 
@@ -29,7 +29,7 @@ EXPORTS = (
     "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
     "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulator_workspace_bytes", "placeto_simulate_runtime",
-    "placeto_policy_gradient", "placeto_last_launch_count",
+    "placeto_policy_gradient", "placeto_last_launch_count", "placeto_last_status", "placeto_debug_wait_timeout",
 )
 
 
@@ -77,7 +77,8 @@ def _load() -> ctypes.CDLL:
     for name in ("placeto_graph_create", "placeto_graph_info", "placeto_graph_host_view",
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
-                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime", "placeto_policy_gradient"):
+                 "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime", "placeto_policy_gradient",
+                 "placeto_last_status", "placeto_debug_wait_timeout"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -402,6 +403,18 @@ def placeto_policy_gradient(g: Graph, w: Weights, X, H_down, H_up, cur, actions,
                                         _stream(stream)),
            "placeto_policy_gradient")
     return grads
+
+
+def placeto_last_status(g: Graph, ws=None, stream=None) -> int:
+    """Status the kernels of the latest call on `g` reported (0 = ok, 8 = a bounded wait ran
+    out); synchronises the stream. `ws`: that call's workspace, None after the _static call."""
+    return int(_lib.placeto_last_status(g.handle, _p(ws), _stream(stream)))
+
+
+def placeto_debug_wait_timeout(g: Graph, ws, stream=None) -> None:
+    """Launches the kernel whose wait is built to run out (tests of the error channel)."""
+    _check(_lib.placeto_debug_wait_timeout(g.handle, _p(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "placeto_debug_wait_timeout")
 
 
 def placeto_last_launch_count() -> int:

@@ -2,9 +2,11 @@
 // layout, schedule selection and kernel launches. No arithmetic of the policy
 // happens on the host.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "kernels.cuh"
 #include "plan.h"
@@ -17,10 +19,12 @@ struct placeto_graph {
     int device = -1;
     DeviceInfo info{};
     int *d_ints = nullptr;       // one allocation for all int arrays
+    int4 *d_packed = nullptr;    // per direction lvl4[n_levels], pos4[n] (see DevLevels)
     int *d_child_ptr = nullptr, *d_child = nullptr, *d_n_parents = nullptr;   // inside d_ints
     int *d_parent_ptr = nullptr, *d_parent = nullptr;                          // inside d_ints
     uint8_t *d_relation = nullptr;
     DevLevels lv[2]{};
+    mutable std::atomic<int> calls{0};   // number of the latest forward call (see StatusSlot)
 };
 
 namespace placeto {
@@ -31,6 +35,7 @@ void count_launch(int k) { t_launches += k; }
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr size_t kStatusBytes = 256;   // reserved at offset 0 of every workspace; the first 4 bytes are the status word
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -76,6 +81,7 @@ placeto_status pool_weights_ok(const placeto_weights *w) {
 }
 
 struct Layout {
+    size_t status;                 // 256 bytes at the start: the status word of the call
     size_t msg[2], msg_alt[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
     int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
@@ -87,6 +93,7 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
     const size_t n = (size_t)g->host.n, d = (size_t)w->d, F = (size_t)w->F, m = (size_t)w->m;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.status = take(kStatusBytes);
     int chunks = pool_chunks((int)n, B, g->info);
     L.chunk_nodes = ((int)n + chunks - 1) / chunks;
     L.chunks = ((int)n + L.chunk_nodes - 1) / L.chunk_nodes;
@@ -146,7 +153,7 @@ unsigned pick_schedule(unsigned flags) {
 
 bool flags_ok(uint32_t flags) {
     const uint32_t known = PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE |
-                           PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR;
+                           PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR | PLACETO_TCGEN05;
     if (flags & ~known) return false;
     const uint32_t sched = flags & (PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE);
     return (sched & (sched - 1)) == 0;   // at most one schedule
@@ -163,6 +170,15 @@ const void *device_alias(const void *p) {
     return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
 }
 
+// The report slot of a new call on `g`: the record at the start of the workspace (or of the
+// built-in scratch) tagged with the call's number.
+StatusSlot new_status_slot(const placeto_graph *g, char *ws, const Layout &L) {
+    StatusSlot s;
+    s.record = reinterpret_cast<int4 *>(ws + L.status);
+    s.call = g->calls.fetch_add(1) + 1;
+    return s;
+}
+
 placeto_status cuda_status(cudaError_t e) {
     if (e == cudaSuccess) return PLACETO_OK;
     if (e == cudaErrorCooperativeLaunchTooLarge) return PLACETO_ERR_UNSUPPORTED;
@@ -171,8 +187,9 @@ placeto_status cuda_status(cudaError_t e) {
 
 placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const float *X, int B,
                          float *H_down, float *H_up, char *ws, const Layout &L, uint32_t flags,
-                         cudaStream_t stream, bool after_own_kernel = false) {
+                         cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false) {
     EmbedArgs a;
+    a.status = status;
     a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
     a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
     a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
@@ -183,6 +200,11 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
     a.max_level_width = g->host.max_level_width;
     const unsigned schedule = pick_schedule(flags);
+    if ((flags & PLACETO_TCGEN05) && !(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) &&
+        schedule == PLACETO_SLICED && embed_tc_applicable(a)) {
+        cudaError_t e = launch_embed_tc(a, g->info, stream, after_own_kernel);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     const bool want_mma = (flags & PLACETO_TENSOR) ? embed_mma_applicable(a) : embed_mma_preferred(a);
     if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) && schedule == PLACETO_SLICED && want_mma) {
         cudaError_t e = launch_embed_mma(a, g->info, stream, after_own_kernel);
@@ -202,8 +224,9 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
 placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const float *X,
                         const float *H_down, const float *H_up, const int32_t *cur, int B,
                         float *logits, float *probs, char *ws, const Layout &L, uint32_t flags,
-                        cudaStream_t stream, bool after_own_kernel = false) {
+                        cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false) {
     PoolArgs a;
+    a.status = status;
     for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
     a.head = to_dev(w->head);
     a.X = X; a.H[0] = H_down; a.H[1] = H_up;
@@ -224,9 +247,17 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     return cuda_status(launch_policy_generic(a, g->info, stream));
 }
 
+// The graph's arrays, the caller's buffers and the launch all belong to one device: the one
+// that was current at placeto_graph_create must be current again.
+bool on_graph_device(const placeto_graph *g) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == g->device;
+}
+
 placeto_status common_checks(const placeto_graph *g, int32_t B, const void *ws, size_t ws_bytes,
                              size_t need, uint32_t flags) {
     if (!g || !g->on_device || B < 1 || !flags_ok(flags)) return PLACETO_ERR_INVALID_ARG;
+    if (!on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
     if ((size_t)B * g->host.n > (size_t)1 << 31) return PLACETO_ERR_UNSUPPORTED;
     if (!ws || !aligned16(ws)) return PLACETO_ERR_INVALID_ARG;
     if (ws_bytes < need) return PLACETO_ERR_WORKSPACE;
@@ -278,6 +309,7 @@ const char *placeto_status_string(placeto_status s) {
         case PLACETO_ERR_CUDA: return "CUDA error";
         case PLACETO_ERR_NO_MEMORY: return "out of memory";
         case PLACETO_ERR_SCRATCH_LIMIT: return "batch exceeds the built-in scratch of the no-allocation call";
+        case PLACETO_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     }
     return "unknown status";
 }
@@ -295,6 +327,7 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
 
     auto fail = [&](placeto_status st) {
         if (g->d_ints) cudaFree(g->d_ints);
+        if (g->d_packed) cudaFree(g->d_packed);
         if (g->d_relation) cudaFree(g->d_relation);
         delete g;
         return st;
@@ -355,6 +388,32 @@ placeto_status placeto_graph_create(int32_t n, int64_t n_edges, const int32_t *s
     if (cudaMemcpy(g->d_relation, g->host.relation.data(), g->host.relation.size(),
                    cudaMemcpyHostToDevice) != cudaSuccess)
         return fail(PLACETO_ERR_CUDA);
+    {   // packed per-level and per-position records (kernels that stream the schedule)
+        std::vector<int4> packed;
+        size_t at[2][2];
+        for (int dir = 0; dir < 2; ++dir) {
+            const LevelPlan &p = g->host.dir[dir];
+            at[dir][0] = packed.size();
+            int max_nbr = 0;
+            for (int l = 0; l < p.n_levels; ++l) {
+                const int p0 = p.level_ptr[l], p1 = p.level_ptr[l + 1];
+                const int e0 = p.nbr_ptr[p0], e1 = p.nbr_ptr[p1];
+                packed.push_back(make_int4(p0, p1 - p0, e0, e1 - e0));
+                max_nbr = std::max(max_nbr, e1 - e0);
+            }
+            at[dir][1] = packed.size();
+            for (int q = 0; q < g->host.n; ++q)
+                packed.push_back(make_int4(p.nbr_ptr[q], p.nbr_ptr[q + 1], p.own_slot[q], p.order[q]));
+            g->lv[dir].max_level_nbr = max_nbr;
+        }
+        if (cudaMalloc(&g->d_packed, packed.size() * sizeof(int4)) != cudaSuccess) return fail(PLACETO_ERR_NO_MEMORY);
+        if (cudaMemcpy(g->d_packed, packed.data(), packed.size() * sizeof(int4), cudaMemcpyHostToDevice) != cudaSuccess)
+            return fail(PLACETO_ERR_CUDA);
+        for (int dir = 0; dir < 2; ++dir) {
+            g->lv[dir].lvl4 = g->d_packed + at[dir][0];
+            g->lv[dir].pos4 = g->d_packed + at[dir][1];
+        }
+    }
     g->on_device = true;
     *out = g;
     return PLACETO_OK;
@@ -399,6 +458,7 @@ void placeto_graph_destroy(placeto_graph *g) {
         cudaGetDevice(&prev);
         if (prev != g->device) cudaSetDevice(g->device);
         cudaFree(g->d_ints);
+        cudaFree(g->d_packed);
         cudaFree(g->d_relation);
         if (prev != g->device && prev >= 0) cudaSetDevice(prev);
     }
@@ -428,6 +488,8 @@ placeto_status placeto_build_features(const placeto_graph *g, const float *cost,
                                       void *stream) {
     t_launches = 0;
     if (!g || !g->on_device || B < 1 || m < 1 || m > PLACETO_MAX_M) return PLACETO_ERR_INVALID_ARG;
+    if (!on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
+    g->calls.fetch_add(1);
     if (!cost || !bytes || !dev || !cur || !placed || !X) return PLACETO_ERR_INVALID_ARG;
     if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(cur) ||
         !aligned16(placed) || !aligned16(X))
@@ -450,8 +512,9 @@ placeto_status placeto_embed_forward(const placeto_graph *g, const placeto_weigh
     if (s != PLACETO_OK) return s;
     if (!X || !H_down || !H_up || !aligned16(X) || !aligned16(H_down) || !aligned16(H_up))
         return PLACETO_ERR_INVALID_ARG;
-    return run_embed(g, w, X, B, H_down, H_up, static_cast<char *>(workspace), L, flags,
-                     static_cast<cudaStream_t>(stream));
+    char *ws = static_cast<char *>(workspace);
+    return run_embed(g, w, X, B, H_down, H_up, ws, L, flags, static_cast<cudaStream_t>(stream),
+                     new_status_slot(g, ws, L));
 }
 
 placeto_status placeto_policy_logits(const placeto_graph *g, const placeto_weights *w,
@@ -471,8 +534,9 @@ placeto_status placeto_policy_logits(const placeto_graph *g, const placeto_weigh
     if (!aligned16(X) || !aligned16(H_down) || !aligned16(H_up) || !aligned16(cur) ||
         !aligned16(logits) || (probs && !aligned16(probs)))
         return PLACETO_ERR_INVALID_ARG;
-    return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, static_cast<char *>(workspace),
-                    L, flags, static_cast<cudaStream_t>(stream));
+    char *ws = static_cast<char *>(workspace);
+    return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, ws, L, flags,
+                    static_cast<cudaStream_t>(stream), new_status_slot(g, ws, L));
 }
 
 placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weights *w,
@@ -498,11 +562,12 @@ placeto_status placeto_policy_forward(const placeto_graph *g, const placeto_weig
     float *X = reinterpret_cast<float *>(ws + L.X);
     float *Hd = reinterpret_cast<float *>(ws + L.H[0]);
     float *Hu = reinterpret_cast<float *>(ws + L.H[1]);
+    const StatusSlot status = new_status_slot(g, ws, L);
     s = cuda_status(launch_features(g->host.n, B, w->m, cost, bytes, dev, cur, placed, X, st));
     if (s != PLACETO_OK) return s;
-    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, status, true);
     if (s != PLACETO_OK) return s;
-    return run_pool(g, w, X, Hd, Hu, cur, B, logits, probs, ws, L, flags, st, true);
+    return run_pool(g, w, X, Hd, Hu, cur, B, logits, probs, ws, L, flags, st, status, true);
 }
 
 placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto_weights *w,
@@ -562,9 +627,10 @@ placeto_status placeto_policy_forward_host(const placeto_graph *g, const placeto
     s = cuda_status(launch_features(g->host.n, B, w->m, d_cost, d_bytes, d_dev, d_cur, d_placed, X, st,
                                     in_mapped));
     if (s != PLACETO_OK) return s;
-    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, true);
+    const StatusSlot status = new_status_slot(g, ws, L);
+    s = run_embed(g, w, X, B, Hd, Hu, ws, L, flags, st, status, true);
     if (s != PLACETO_OK) return s;
-    s = run_pool(g, w, X, Hd, Hu, d_cur, B, out_logits, out_probs, ws, L, flags, st, true);
+    s = run_pool(g, w, X, Hd, Hu, d_cur, B, out_logits, out_probs, ws, L, flags, st, status, true);
     if (s != PLACETO_OK) return s;
     if (!out_mapped) {
         if (cudaMemcpyAsync(logits, d_logits, mB, cudaMemcpyDeviceToHost, st) != cudaSuccess)
@@ -584,9 +650,9 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
     if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
     placeto_status s = pool_weights_ok(w);
     if (s != PLACETO_OK) return s;
-    if (B < 1 || !flags_ok(flags)) return PLACETO_ERR_INVALID_ARG;
+    if (B < 1 || !flags_ok(flags) || !on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
     if ((size_t)B * g->host.n > (size_t)1 << 31) return PLACETO_ERR_UNSUPPORTED;
-    const Layout L = make_layout(g, w, B, PLACETO_CALL_LOGITS);   // partial sums sit at offset 0
+    const Layout L = make_layout(g, w, B, PLACETO_CALL_LOGITS);   // status record, then the partial sums
     if (L.total > PLACETO_STATIC_SCRATCH_BYTES) return PLACETO_ERR_SCRATCH_LIMIT;
     if (!X || !H_down || !H_up || !cur || !logits) return PLACETO_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(H_down) || !aligned16(H_up) || !aligned16(cur) ||
@@ -595,7 +661,7 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
     char *scratch = static_scratch_address(g->device);
     if (!scratch) return PLACETO_ERR_CUDA;
     return run_pool(g, w, X, H_down, H_up, cur, B, logits, probs, scratch, L, flags,
-                    static_cast<cudaStream_t>(stream));
+                    static_cast<cudaStream_t>(stream), new_status_slot(g, scratch, L));
 }
 
 placeto_status placeto_embed_rounds(const placeto_graph *g, const placeto_weights *w, const float *X,
@@ -606,6 +672,7 @@ placeto_status placeto_embed_rounds(const placeto_graph *g, const placeto_weight
     placeto_status s = embed_weights_ok(w);
     if (s != PLACETO_OK) return s;
     if (B < 1 || rounds < 0) return PLACETO_ERR_INVALID_ARG;
+    g->calls.fetch_add(1);
     const Layout L = make_layout(g, w, B, PLACETO_CALL_EMBED_ROUNDS);
     s = common_checks(g, B, workspace, workspace_bytes, L.total, 0);
     if (s != PLACETO_OK) return s;
@@ -669,15 +736,16 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
     ep.logp = logp; ep.actions = actions;
     float *probs = reinterpret_cast<float *>(ws + L.probs);
     ep.X = X;
+    const StatusSlot status = new_status_slot(g, ws, L);
     s = cuda_status(launch_episode_begin(ep, st));
     // the features of the initial states; every later step patches them in place
     if (s == PLACETO_OK)
         s = cuda_status(launch_features(ep.n, E, w->m, cost, bytes, dev, ep.cur, ep.placed, X, st));
     for (int t = 0; s == PLACETO_OK && t < ep.n; ++t) {
         // one policy evaluation of the E current states, then the transition
-        s = run_embed(g, w, X, E, Hd, Hu, ws, L, flags, st, true);
+        s = run_embed(g, w, X, E, Hd, Hu, ws, L, flags, st, status, true);
         if (s == PLACETO_OK)
-            s = run_pool(g, w, X, Hd, Hu, ep.cur, E, const_cast<float *>(ep.logits), probs, ws, L, flags, st, true);
+            s = run_pool(g, w, X, Hd, Hu, ep.cur, E, const_cast<float *>(ep.logits), probs, ws, L, flags, st, status, true);
         if (s == PLACETO_OK) s = cuda_status(launch_episode_step(ep, t, st));
     }
     return s;
@@ -694,7 +762,8 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
                                         void *stream) {
     t_launches = 0;
     if (!g || !g->on_device || P < 1 || m < 1 || m > PLACETO_MAX_M) return PLACETO_ERR_INVALID_ARG;
-    if (!(bandwidth > 0.0)) return PLACETO_ERR_INVALID_ARG;
+    if (!(bandwidth > 0.0) || !on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
+    g->calls.fetch_add(1);
     if (!cost || !bytes || !dev || !runtime || !workspace) return PLACETO_ERR_INVALID_ARG;
     if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(runtime) ||
         !aligned16(workspace))
@@ -723,6 +792,7 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
     if (s == PLACETO_OK) s = pool_weights_ok(w);
     if (s != PLACETO_OK) return s;
     if (B < 1 || !grads) return PLACETO_ERR_INVALID_ARG;
+    g->calls.fetch_add(1);
     // the gradient buffers mirror the weights' shapes
     if (grads->d != w->d || grads->F != w->F || grads->m != w->m) return PLACETO_ERR_INVALID_ARG;
     const placeto_mlp *wn[11] = {&w->f_down, &w->f_up, &w->g_down, &w->g_up, &w->l[0], &w->l[1], &w->l[2],
@@ -772,6 +842,31 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
     a.ghead = out(grads->head);
     return cuda_status(launch_policy_gradient(a, g->info, static_cast<float *>(workspace),
                                               static_cast<cudaStream_t>(stream)));
+}
+
+placeto_status placeto_last_status(const placeto_graph *g, const void *workspace, void *stream) {
+    if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
+    const char *at = static_cast<const char *>(workspace);
+    if (!at) {
+        at = static_scratch_address(g->device);
+        if (!at) return PLACETO_ERR_CUDA;
+    }
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PLACETO_ERR_CUDA;
+    int rec[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(rec, at, sizeof(rec), cudaMemcpyDeviceToHost) != cudaSuccess) return PLACETO_ERR_CUDA;
+    if (rec[0] != kStatusMagic0 || rec[1] != kStatusMagic1 || rec[2] != g->calls.load()) return PLACETO_OK;
+    return rec[3] > 0 && rec[3] <= PLACETO_ERR_TIMEOUT ? static_cast<placeto_status>(rec[3]) : PLACETO_ERR_CUDA;
+}
+
+placeto_status placeto_debug_wait_timeout(const placeto_graph *g, void *workspace, size_t workspace_bytes,
+                                          void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device || !workspace || !aligned16(workspace)) return PLACETO_ERR_INVALID_ARG;
+    if (!on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
+    if (workspace_bytes < kStatusBytes) return PLACETO_ERR_WORKSPACE;
+    Layout L{};
+    return cuda_status(launch_wait_timeout_probe(new_status_slot(g, static_cast<char *>(workspace), L),
+                                                 static_cast<cudaStream_t>(stream)));
 }
 
 int32_t placeto_last_launch_count(void) { return t_launches; }

@@ -1,5 +1,5 @@
 // Gradient of the policy objective with respect to every weight (Appendix A.1
-// and A.6 of the Placeto paper: the REINFORCE term sum_b A_b log pi(a_b | s_b)
+// and A.7 of the Placeto paper: the REINFORCE term sum_b A_b log pi(a_b | s_b)
 // plus an entropy term beta sum_b H(pi(. | s_b))), by reverse-mode
 // differentiation of the forward path:
 //

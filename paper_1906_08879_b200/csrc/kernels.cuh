@@ -18,6 +18,11 @@ struct DevLevels {
     int n_slots;                     // on-chip message slots (see plan.h)
     const int *own_slot, *nbr_slot;
     int n_nbr;                       // total neighbour entries
+    // packed records for kernels that stream the schedule level by level:
+    //   lvl4[level] = {first position, width, first neighbour entry, neighbour entries of the level}
+    //   pos4[p]     = {first neighbour entry, end of neighbour entries, own slot, node id}
+    const int4 *lvl4, *pos4;
+    int max_level_nbr;               // most neighbour entries in one level
 };
 
 // One feed-forward network with device pointers.
@@ -45,6 +50,21 @@ inline size_t mlp_floats(const DevMlp &m) {
     return s;
 }
 
+// Where a kernel reports a bounded wait that ran out (or, in a PLACETO_DEBUG build, an index
+// out of range): a 16-byte record {magic, magic, call number, status code}. A record counts
+// only if it carries the number of the call that asks, so nothing ever has to be cleared and
+// whatever an uninitialised workspace holds cannot be mistaken for a report.
+constexpr int kStatusMagic0 = 0x504c4143, kStatusMagic1 = 0x544f5354;
+struct StatusSlot {
+    int4 *record;   // device memory, 16-byte aligned (null: nowhere to report)
+    int call;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ void report_status(const StatusSlot &s, int code) {
+    if (s.record != nullptr) *s.record = make_int4(kStatusMagic0, kStatusMagic1, s.call, code);
+}
+#endif
+
 struct EmbedArgs {
     DevLevels lv[2];
     DevMlp f[2], g[2];
@@ -53,6 +73,7 @@ struct EmbedArgs {
     float *M[2];   // messages f([h || x]) per node and state, [n][B][d] (workspace)
     int n, B, F, d;
     int max_level_width;   // widest level over both directions
+    StatusSlot status;
 };
 
 struct PoolArgs {
@@ -64,6 +85,7 @@ struct PoolArgs {
     float *logits, *probs;     // [B][m]; probs may be null
     int n, B, F, d, m;
     int chunks, chunk_nodes;
+    StatusSlot status;
 };
 
 struct EpisodeArgs {
@@ -241,6 +263,17 @@ bool embed_mma_applicable(const EmbedArgs &a);
 bool embed_mma_preferred(const EmbedArgs &a);   // applicable and faster than the FMA kernels
 cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
                              bool overlap = false);
+
+// embed_tc.cu: d = 64 on tcgen05 tensor cores with accumulators in tensor memory (TF32 head + tail
+// operands, all four partial products per instruction). A bounded wait that runs out inside the
+// kernel is reported through a.status as PLACETO_ERR_TIMEOUT.
+bool embed_tc_applicable(const EmbedArgs &a);
+cudaError_t launch_embed_tc(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap = false);
+
+// A kernel whose only job is to let a bounded wait run out (a copy that delivers fewer bytes
+// than the barrier expects, a poll limit of a few thousand tries) and report it: exercises the
+// time-out path without faulting or hanging anything.
+cudaError_t launch_wait_timeout_probe(const StatusSlot &status, cudaStream_t stream);
 
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);

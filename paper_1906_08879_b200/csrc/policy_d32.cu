@@ -106,6 +106,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
         else bulk_load(xs + (size_t)q * kWarps * FP, a.X + row * F, x_bytes, &bar);
     }
     const bool landed = mbar_wait(&bar, 0);
+    if (!landed && threadIdx.x == 0) report_status(a.status, PLACETO_ERR_TIMEOUT);
 
     if (warp >= nb) return;
     const int b = b0 + warp;

@@ -158,6 +158,7 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     };
     load_set(0);
     const bool landed = mbar_wait(&bar, 0);
+    if (!landed && threadIdx.x == 0) report_status(a.status, PLACETO_ERR_TIMEOUT);
     __syncthreads();            // lists, counts and the zero padding written by other threads
 
     for (int i = 0; i < 3; ++i) {

@@ -1,5 +1,5 @@
 // Run time of a placement under the event-based execution model of the Placeto
-// paper's simulator (Appendix A.4): every device runs one operation at a time
+// paper's simulator (Appendix A.5): every device runs one operation at a time
 // from a FIFO queue of runnable operations; every device's bus sends one output
 // tensor at a time from a FIFO queue, overlapping with compute; an operation is
 // runnable once all parents have finished and their outputs have arrived on its

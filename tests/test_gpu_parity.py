@@ -29,7 +29,8 @@ TOL_ELEM, TOL_NORM = 1e-4, 2e-5
 SCHEDULES = {"sliced": placeto.PLACETO_SLICED, "per_level": placeto.PLACETO_PER_LEVEL,
              "cooperative": placeto.PLACETO_COOPERATIVE,
              "generic_sliced": placeto.PLACETO_SLICED | placeto.PLACETO_GENERIC,
-             "fma_only": placeto.PLACETO_FMA_ONLY, "tensor": placeto.PLACETO_TENSOR}
+             "fma_only": placeto.PLACETO_FMA_ONLY, "tensor": placeto.PLACETO_TENSOR,
+             "tcgen05": placeto.PLACETO_TCGEN05}
 
 
 def dev_t(a):
@@ -124,27 +125,41 @@ def test_nmt(normalise, flags):
     compare(cfg, out, oracle.forward(cfg, threads=8))
 
 
-@pytest.mark.parametrize("flags", [0, placeto.PLACETO_FMA_ONLY])
+@pytest.mark.parametrize("flags", [0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TCGEN05])
 def test_nasnet_full_batch_sampled_states(flags):
     """Full size on the GPU (n ~ 2100, B = 512, d = 64); the checker evaluates
-    a sample of states one by one (states are independent)."""
+    a sample of states one by one (states are independent). At this batch the
+    tensor-core kernels give a block a slice of 8 (mma.sync) or 7 (tcgen05)
+    states that share the rows of a tile: the sample holds every position of a
+    slice (states 0..7 and 504..511 under either slicing) and states from the
+    middle of the batch."""
     cfg = configs.make("nasnet")
     out = gpu_forward(cfg, flags)
-    sel = np.asarray([0, 1, 63, 64, 255, 256, 300, 448, 510, 511])
+    sel = np.asarray(list(range(8)) + [63, 64, 255, 258, 259, 261, 300, 448] + list(range(504, 512)))
     compare(cfg, out, oracle.forward(cfg, threads=8, states=sel), sel=sel)
     for k in ("H_down", "H_up", "logits", "probs"):
         assert torch.isfinite(out[k]).all()
 
 
-@pytest.mark.parametrize("flags", [0, placeto.PLACETO_TENSOR])
-@pytest.mark.parametrize("i", [0, 1, 30, 63])
-def test_episode_sweep(i, flags):
+def _sweep_case(i, flags, samples):
     cfg = configs.make_sweep(i)
     out = gpu_forward(cfg, flags)
     n = cfg["n"]
-    sel = None if n <= 320 else np.unique(np.linspace(0, n - 1, 48).astype(int))
+    sel = None if n <= 320 else np.unique(np.linspace(0, n - 1, samples).astype(int))
     ref = oracle.forward(cfg, threads=8, states=sel)
     compare(cfg, out, ref, sel=sel)
+
+
+@pytest.mark.parametrize("i", range(64))
+def test_episode_sweep(i):
+    """Every graph of the full-episode sweep, all |V| states on the GPU; the
+    checker takes all of them up to 320 nodes and 24 evenly spaced ones beyond."""
+    _sweep_case(i, 0, 24)
+
+
+@pytest.mark.parametrize("i", [0, 1, 30, 63])
+def test_episode_sweep_on_the_tensor_kernel(i):
+    _sweep_case(i, placeto.PLACETO_TENSOR, 48)
 
 
 # ------------------------------------------------------------- edge cases ---
@@ -198,8 +213,79 @@ def test_specialised_kernels_over_feature_widths(d, m):
     n = int(r.integers(30, 90))
     src, dst = random_dag(r, n, float(r.uniform(0.03, 0.12)))
     B = int(r.integers(3, 70))
-    for flags in (0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR):
+    for flags in (0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR, placeto.PLACETO_TCGEN05):
         _small_case(n, src, dst, d=d, m=m, B=B, seed=m + d, schedule=flags)
+
+
+@pytest.mark.parametrize("B", [1, 7, 33, 300, 1200])
+def test_tcgen05_kernel_over_batch_sizes(B):
+    """d = 64 on tcgen05: one state per block, ragged last slice, slices of up to
+    17 states (tiles of more than 32 and more than 64 rows on the wide levels)."""
+    r = rng(B)
+    src, dst = random_dag(r, 60, 0.08)
+    _small_case(60, src, dst, d=64, m=8, B=B, seed=B, schedule=placeto.PLACETO_TCGEN05)
+
+
+def test_tcgen05_kernel_on_a_deep_chain_and_a_wide_level():
+    n = 1500
+    src = list(range(n - 1)) + list(range(0, n - 40, 37))
+    dst = list(range(1, n)) + [i + 40 for i in range(0, n - 40, 37)]
+    _small_case(n, src, dst, d=64, m=8, B=10, seed=29, schedule=placeto.PLACETO_TCGEN05)
+    # 40 roots -> 12 nodes -> 1 sink with 20 states per block: levels of 800 and 240 rows
+    r = rng(31)
+    src = list(range(40)) + [40 + i for i in range(12)]
+    dst = [40 + int(r.integers(0, 12)) for _ in range(40)] + [52] * 12
+    _small_case(53, src, dst, d=64, m=12, B=1480, seed=31, schedule=placeto.PLACETO_TCGEN05)
+
+
+def test_error_channel_reports_a_wait_that_ran_out():
+    """A kernel whose barrier can never complete gives up after a bounded number of
+    polls and reports it; the record is tied to its call, so the next call (and
+    a workspace full of whatever memory held before) reads as clean. Nothing
+    faults: the same context carries on."""
+    cfg = configs.make("tiny")
+    g = placeto.Graph(cfg["n"], cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    ws = placeto.workspace(g, w, cfg["B"], placeto.CALL_FORWARD)
+    ws.fill_(0xAB)
+    assert placeto.placeto_last_status(g, ws) == 0
+    placeto.placeto_debug_wait_timeout(g, ws)
+    assert placeto.placeto_last_status(g, ws) == 8
+    assert placeto.binding.status_string(8) == "a bounded wait inside a kernel ran out"
+    out = gpu_forward(cfg)
+    compare(cfg, out, oracle.forward(cfg))
+    logits, _ = placeto.placeto_policy_forward(g, w, dev_t(cfg["cost"]), dev_t(cfg["bytes"]), dev_t(cfg["dev"]),
+                                               dev_t(cfg["cur"]), dev_t(cfg["placed"]), ws=ws)
+    assert placeto.placeto_last_status(g, ws) == 0
+    assert torch.equal(logits, out["logits"])
+
+
+@pytest.mark.parametrize("name", ["tiny", "inception", "nmt", "nasnet", "sweep63"])
+def test_error_at_the_one_percent_floor_beside_the_single_precision_checker(name, capsys):
+    """The gates above put the floor of the elementwise error at 0.1 of the row's
+    largest entry. With the floor at 0.01 the error of ANY fp32 evaluation grows
+    (small entries of a row carry the row's absolute error): the library's figure
+    is reported beside that of the checker compiled in single precision and held
+    to three times it."""
+    cfg = configs.make_sweep(63) if name == "sweep63" else configs.make(name)
+    B = cfg["B"]
+    sel = None if B <= 16 else np.unique(np.linspace(0, B - 1, 16).astype(int))
+    out = gpu_forward(cfg)
+    ref = oracle.forward(cfg, threads=8, states=sel)
+    can = oracle.forward(cfg, real="float", threads=8, states=sel)
+    worst = 0.0
+    lines = []
+    for key in ("H_down", "H_up", "logits"):
+        got = out[key].cpu().numpy()
+        if sel is not None:
+            got = got[:, sel] if key != "logits" else got[sel]
+        e_gpu = row_rel_err(got, ref[key], 0.01)
+        e_can = row_rel_err(can[key], ref[key], 0.01)
+        lines.append("%s %s: library %.3g, single-precision checker %.3g" % (name, key, e_gpu, e_can))
+        worst = max(worst, e_gpu / max(3.0 * e_can, 1e-5))
+    with capsys.disabled():
+        print("\n[0.01 floor] " + "; ".join(lines))
+    assert worst <= 1.0, lines
 
 
 def test_single_layer_networks_as_in_the_paper():
