@@ -5,8 +5,10 @@
 
 A step is one pass of the whole path (features -> two-way message passing ->
 group pooling -> head -> softmax) over one batch of synthetic placement states
-through the C ABI. The default workload is the Inception-shaped configuration
-(~300 nodes, d = 32, 256 states). Prints one JSON line.
+through the C ABI. The default workload is the NASNet-shaped configuration, the
+largest of the five (2130 nodes in 744 levels, d = 64, 512 states); the same line
+carries short measurements of the other four under "other_workloads" and the
+library's error against the CPU checker on a sample of states. Prints one JSON line.
 
 Multi-GPU (torchrun, one rank per GPU): states are independent, so every rank
 runs its own batch of the same size (weak scaling) with no data-path
@@ -40,8 +42,10 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="inception",
-                    help="tiny | inception | nmt | nasnet | sweepNN")
+    ap.add_argument("--workload", default="nasnet",
+                    help="tiny | inception | nmt | nasnet | nasnet_wide | sweepNN")
+    ap.add_argument("--no-others", action="store_true",
+                    help="skip the short measurements of the other workloads (other_workloads)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--flags", type=int, default=0, help="schedule flags of placeto.h")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0)
@@ -242,6 +246,80 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ B200 ----
 
+def error_against_checker(cfg, logits, Hd, Hu, samples: int = 16):
+    """The library's outputs against the CPU checker on evenly spaced states:
+    elementwise error with the floor at 0.1 and at 0.01 of the row's largest
+    entry, normwise error, and decisive states whose argmax differs."""
+    from oracle import oracle
+    B = cfg["B"]
+    sel = np.arange(B) if B <= samples else np.unique(np.linspace(0, B - 1, samples).astype(int))
+    ref = oracle.forward(cfg, threads=len(os.sched_getaffinity(0)), states=sel)
+
+    def err(got, want, floor):
+        row = np.max(np.abs(want), axis=-1, keepdims=True)
+        den = np.maximum(np.abs(want), floor * row)
+        den = np.where(den == 0, 1.0, den)
+        return float(np.max(np.abs(got.astype(np.float64) - want) / den))
+
+    got = {"H_down": Hd[:, sel].cpu().numpy(), "H_up": Hu[:, sel].cpu().numpy(), "logits": logits[sel].cpu().numpy()}
+    srt = np.sort(ref["logits"], axis=1)
+    gap = srt[:, -1] - srt[:, -2] if srt.shape[1] > 1 else np.full(len(srt), np.inf)
+    decisive = gap > np.maximum(1e-3, 2e-5 * np.abs(ref["logits"]).max(axis=1))
+    differ = got["logits"].argmax(axis=1) != ref["logits"].argmax(axis=1)
+    return {"states_checked": int(len(sel)),
+            "max_rel_err": max(err(got[k], ref[k], 0.1) for k in got),
+            "max_rel_err_floor_0p01": max(err(got[k], ref[k], 0.01) for k in got),
+            "max_norm_err": max(err(got[k], ref[k], 1.0) for k in got),
+            "argmax_mismatches": int((differ & decisive).sum()), "decisive_states": int(decisive.sum()),
+            "reference": "fp64 CPU checker (oracle/), same seeded inputs"}
+
+
+def measure_workload(name: str, steps: int, warmup: int, flags: int, sm_count: int, peak_tflops: float):
+    """Short measurement of one workload on the current device: whole path and
+    the message-passing launch alone, L2 flushed before every timed call."""
+    import torch
+    import paper_1906_08879_b200 as placeto
+    cfg = make_workload(name)
+    n, B, m, d, F = cfg["n"], cfg["B"], cfg["m"], cfg["d"], cfg["F"]
+    g = placeto.Graph(n, cfg["src"], cfg["dst"])
+    w = placeto.Weights(cfg["weights"])
+    dev_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    cost, nbytes = dev_t(cfg["cost"]), dev_t(cfg["bytes"])
+    devs, cur, placed = dev_t(cfg["dev"]), dev_t(cfg["cur"]), dev_t(cfg["placed"])
+    logits = torch.empty((B, m), dtype=torch.float32, device="cuda")
+    probs = torch.empty((B, m), dtype=torch.float32, device="cuda")
+    ws = placeto.workspace(g, w, B, placeto.CALL_FORWARD, flags)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    X = placeto.placeto_build_features(g, cost, nbytes, devs, cur, placed, m)
+    Hd = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
+    Hu = torch.empty((n, B, d), dtype=torch.float32, device="cuda")
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(steps):
+            flush.zero_()
+            starts[i].record(stream)
+            fn()
+            ends[i].record(stream)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in zip(starts, ends)) / steps
+
+    step_ms = timed(lambda: placeto.placeto_policy_forward(g, w, cost, nbytes, devs, cur, placed, logits, probs,
+                                                           ws, flags, stream))
+    embed_ms = timed(lambda: placeto.placeto_embed_forward(g, w, X, Hd, Hu, ws, flags, stream))
+    achieved = flops_embed(cfg) / (embed_ms * 1e-3) / 1e12
+    out = {"n_nodes": n, "depth": cfg["depth"], "d": d, "states": B, "ms_per_step": step_ms,
+           "value": B / (step_ms * 1e-3), "embed_ms": embed_ms,
+           "roofline_frac": achieved / peak_tflops if d >= 32 else None}
+    out.update(error_against_checker(cfg, logits, Hd, Hu))
+    del out["reference"]
+    return out
+
+
 def run_b200(args):
     import torch
     import paper_1906_08879_b200 as placeto
@@ -410,8 +488,10 @@ def run_b200(args):
                            if args.rounds > 0 else "message passing (embed_forward, %d launch(es))" % embed_launches),
                 "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved / peak_tflops,
                 "traffic": traffic, "traffic_source": traffic_from,
-                "arithmetic": ("fp32 accumulate on mma.sync, TF32 head+tail operands (3 products)"
-                               if d == 64 and not (args.flags & 16) else "fp32 fma"),
+                "arithmetic": ("fp32 accumulate on tcgen05.mma, TF32 head+tail operands (4 products per instruction)"
+                               if d == 64 and (args.flags & 64) and not (args.flags & 24)
+                               else "fp32 accumulate on mma.sync, TF32 head+tail operands (3 products)"
+                               if d == 64 and not (args.flags & 24) else "fp32 fma"),
                 "algorithmic_bytes": (4 * F + 8 * d) * n * B,
                 "hbm": {"achieved": (4 * F + 8 * d) * n * B / (embed_ms * 1e-3) / 1e9, "peak": hbm_peak,
                         "unit": "GB/s", "frac": (4 * F + 8 * d) * n * B / (embed_ms * 1e-3) / 1e9 / hbm_peak,
@@ -425,6 +505,18 @@ def run_b200(args):
     cores = len(os.sched_getaffinity(0))
     cpu_value, cpu_s, passes = time_oracle(cfg, args.cpu_baseline_seconds, cores)
     config = workload_config(cfg, world)
+    parity = None
+    others = None
+    if args.episodes == 0:
+        step()                                        # the outputs of this rank's own batch
+        embed_only()
+        torch.cuda.synchronize()
+        parity = error_against_checker(cfg, logits, Hd, Hu)
+        if world == 1 and not args.no_others and args.rounds == 0:
+            others = {}
+            for other in ("tiny", "inception", "nmt", "sweep63", "nasnet_wide", "nasnet"):
+                if other != cfg["name"] and not (other == "sweep63" and cfg["name"].startswith("sweep")):
+                    others[other] = measure_workload(other, min(args.steps, 30), 3, args.flags, sm_count, peak_tflops)
     if args.episodes > 0:
         config.update(workload=cfg["name"] + "-episodes", episodes_per_gpu=B, steps_per_episode=n,
                       choice="sampled (inverse CDF of the device softmax)",
@@ -438,6 +530,12 @@ def run_b200(args):
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": "%d full passes over the batch of %d states (%.2f s each)"
                                        % (passes, B, cpu_s)}}
+    if parity is not None:
+        line["parity"] = parity
+        for k in ("max_rel_err", "max_norm_err", "argmax_mismatches"):
+            line[k] = parity[k]
+    if others is not None:
+        line["other_workloads"] = others
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

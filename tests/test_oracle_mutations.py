@@ -57,6 +57,12 @@ MUTATIONS = [
      "            memcpy(e, H_up + ((size_t)u * B + b) * d, sizeof(real) * (size_t)d);"),
     ("softmax not normalised", "probs[(size_t)b * m + k] /= tot;", "(void)tot;"),
     ("one-hot off by one", "(dev[(size_t)b * n + v] == k) ? 1 : 0", "(dev[(size_t)b * n + v] == k + 1) ? 1 : 0"),
+    ("synchronous rounds update in place",
+     "memcpy(in, prev + ((size_t)u * B + b) * d, sizeof(real) * (size_t)d);",
+     "memcpy(in, H + ((size_t)u * B + b) * d, sizeof(real) * (size_t)d);"),
+    ("synchronous rounds start from the bias-only state instead of zeros",
+     "for (size_t i = 0; i < tot; ++i) H[i] = 0;\n        for (int r = 0; r < rounds; ++r) {",
+     "for (size_t i = 0; i < tot; ++i) H[i] = 0;\n        for (int r = -1; r < rounds; ++r) {"),
     ("sum over neighbours replaced by the last neighbour", "for (int j = 0; j < d; ++j) s[j] += msg[j];\n        }\n        mlp(gg,",
      "for (int j = 0; j < d; ++j) s[j] = msg[j];\n        }\n        mlp(gg,"),
 ]
@@ -77,6 +83,7 @@ PINS = [
     pins.test_influence_sets,
     lambda: pins.test_brute_force_random_small_dags(5, 1),
     lambda: pins.test_brute_force_random_small_dags(6, 2),
+    lambda: pins.test_synchronous_rounds_truncated_series(2),
 ]
 
 

@@ -232,6 +232,36 @@ def test_synchronous_rounds_reach_progressive_sweep():
     assert not np.array_equal(Sd3, Hd)
 
 
+@pytest.mark.parametrize("layers", [1, 2])
+def test_synchronous_rounds_truncated_series(layers):
+    """Finite k (Sec. 2.2 step 2: the update repeated k times, from zeros). For
+    affine f and g one round is H <- P^T H A + T with T = P^T X C + deg (x) c + 1 (x) b_g,
+    so k rounds give the k-term series  sum_{j<k} (P^T)^j T A^j:  matrix powers,
+    no iteration. Fixes the values at k = 1, 2, 3 (below the depth)."""
+    n, d, m, B = 12, 3, 2, 2
+    F = m + 4
+    r = rng(41)
+    src, dst = random_dag(r, n, 0.3)
+    w = _linear_weights(r, d, F, m, layers)
+    X = r.normal(size=(n, B, F))
+    for k in (0, 1, 2, 3):
+        Sd, Su = oracle.embed_sync(n, src, dst, X, w, rounds=k)
+        for name, S, down in (("down", Sd, True), ("up", Su, False)):
+            Wf, bf = _collapse(w["f_" + name])
+            Wg, bg = _collapse(w["g_" + name])
+            A, C = Wf[:d] @ Wg, Wf[d:] @ Wg
+            P = np.zeros((n, n))
+            for u, v in set(zip(map(int, src), map(int, dst))):
+                P[(u, v) if down else (v, u)] = 1.0
+            deg = P.sum(axis=0)
+            for b in range(B):
+                T = P.T @ X[:, b, :] @ C + np.outer(deg, bf @ Wg) + bg[None, :]
+                want = np.zeros((n, d))
+                for j in range(k):
+                    want += np.linalg.matrix_power(P.T, j) @ T @ np.linalg.matrix_power(A, j)
+                np.testing.assert_allclose(S[:, b, :], want, rtol=1e-10, atol=1e-12)
+
+
 # ---------------------------------------------------- P8: influence sets ---
 
 def test_influence_sets():
