@@ -196,7 +196,12 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         const int e0 = lv.nbr_ptr[i], e1 = lv.nbr_ptr[i + 1];
         const int first = e1 > e0 ? lv.nbr_slot[e0] : 0;
         meta_w[i] = make_int4(e0, e1, (lv.own_slot[i] & 0xffff) | (first << 16), lv.order[i]);
+        PLACETO_DEBUG_CHECK(a.status, e0 >= 0 && e0 <= e1 && e1 <= lv.n_nbr && lv.own_slot[i] >= -1 &&
+                                          lv.own_slot[i] < lv.n_slots && lv.order[i] >= 0 && lv.order[i] < a.n);
     }
+    for (int e = threadIdx.x; e < lv.n_nbr; e += kThreads)
+        PLACETO_DEBUG_CHECK(a.status, lv.nbr_slot[e] >= 0 && lv.nbr_slot[e] < lv.n_slots);
+    PLACETO_DEBUG_CHECK(a.status, nb >= 1 && b_first + nb <= B);
     const int4 *meta = meta_w;
     int *ism = reinterpret_cast<int *>(smem) + 4 * a.n;
     auto stage = [&](const int *src, int count) {

@@ -167,7 +167,15 @@ embed_mma_kernel(const EmbedArgs a, const MmaPlan p) {
     int *ism = reinterpret_cast<int *>(base);
     int4 *meta_w = reinterpret_cast<int4 *>(ism);
     for (int i = gt; i < a.n; i += GT)
+    {
         meta_w[i] = make_int4(lv.nbr_ptr[i], lv.nbr_ptr[i + 1], lv.own_slot[i], lv.order[i]);
+        PLACETO_DEBUG_CHECK(a.status, lv.nbr_ptr[i] >= 0 && lv.nbr_ptr[i] <= lv.nbr_ptr[i + 1] &&
+                                          lv.nbr_ptr[i + 1] <= lv.n_nbr && lv.own_slot[i] >= -1 &&
+                                          lv.own_slot[i] < lv.n_slots && lv.order[i] >= 0 && lv.order[i] < a.n);
+    }
+    for (int e = gt; e < lv.n_nbr; e += GT)
+        PLACETO_DEBUG_CHECK(a.status, lv.nbr_slot[e] >= 0 && lv.nbr_slot[e] < lv.n_slots);
+    PLACETO_DEBUG_CHECK(a.status, nb >= 1 && b_first + nb <= B);
     ism += 4 * a.n;
     auto stage = [&](const int *src, int count) {
         int *dst = ism;

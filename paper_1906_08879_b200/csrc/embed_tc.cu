@@ -477,10 +477,17 @@ __global__ void __launch_bounds__(kThreads, 1) embed_tc_kernel(const EmbedArgs a
             for (int r = lane; r < L.y * nb; r += 32) {
                 const int qp = nb == 1 ? r : (int)__umulhi((unsigned)r, magic_nb), s = r - qp * nb;
                 const int4 m = pos4[L.x + qp];   // neighbour range, own slot, node id
+                PLACETO_DEBUG_CHECK(a.status, m.x >= L.z && m.x <= m.y && m.y <= L.z + L.w && m.z >= -1 &&
+                                                  m.z < lv.n_slots && m.w >= 0 && m.w < a.n && b_first + s < B);
                 rec[r] = make_int4((m.x - L.z) | ((m.y - m.x) << 16), s, m.z >= 0 ? (m.z * S + s) * D : -1,
                                    m.w * B + b_first + s);
             }
-            for (int e = lane; e < L.w; e += 32) nslot[e] = lv.nbr_slot[L.z + e];
+            for (int e = lane; e < L.w; e += 32) {
+                nslot[e] = lv.nbr_slot[L.z + e];
+                PLACETO_DEBUG_CHECK(a.status, nslot[e] >= 0 && nslot[e] < lv.n_slots);
+            }
+            PLACETO_DEBUG_CHECK(a.status, L.x >= 0 && L.y >= 1 && L.x + L.y <= a.n && L.y <= a.max_level_width &&
+                                              L.w <= lv.max_level_nbr);
             if (vec) {
                 const int per4 = per_node >> 2;
                 for (int i = lane; i < L.y * per4; i += 32) {

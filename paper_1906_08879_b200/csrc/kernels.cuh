@@ -63,6 +63,16 @@ struct StatusSlot {
 __device__ __forceinline__ void report_status(const StatusSlot &s, int code) {
     if (s.record != nullptr) *s.record = make_int4(kStatusMagic0, kStatusMagic1, s.call, code);
 }
+// Index checks of a library built with -DPLACETO_DEBUG (the stand-in for a memory checker):
+// a schedule record, slot, node or state index out of range is reported as
+// PLACETO_ERR_INVALID_ARG through the call's status record; nothing traps. The kernels test the
+// records where they stage them, before any access uses them. Without the flag no code is made.
+#ifdef PLACETO_DEBUG
+#define PLACETO_DEBUG_CHECK(status, cond) \
+    do { if (!(cond)) placeto::report_status((status), PLACETO_ERR_INVALID_ARG); } while (0)
+#else
+#define PLACETO_DEBUG_CHECK(status, cond) do { } while (0)
+#endif
 #endif
 
 struct EmbedArgs {

@@ -112,6 +112,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     const int b = b0 + warp;
     const int c = a.cur[b];
     const bool valid = c >= 0 && c < n;
+    PLACETO_DEBUG_CHECK(a.status, valid);
     const uint8_t *rel = a.relation + (size_t)(valid ? c : 0) * n + u0;
     float *out = a.partial + ((size_t)chunk * B + b) * 3 * kD;
     for (int i = 0; i < 3; ++i) {

@@ -129,6 +129,7 @@ pool_d64_kernel(const PoolArgs a, const Pool64Plan p) {
     if (warp < nb) {       // warp s compacts the relation row of its state into three lists
         const int c = a.cur[b0 + warp];
         const bool valid = c >= 0 && c < n;
+    PLACETO_DEBUG_CHECK(a.status, valid);
         const uint8_t *rel = a.relation + (size_t)(valid ? c : 0) * n + u0;
         int cnt[3] = {0, 0, 0};
         for (int base = 0; base < nu; base += 32) {
