@@ -394,6 +394,28 @@ placeto_status placeto_policy_logits_static(const placeto_graph *g, const placet
                                             void *stream);
 
 /*
+ * The "simple aggregator" policy of the paper's ablation (Sec. 4.3, "Alternative policy
+ * architectures", variant 1: one feed-forward network aggregates all the node features of
+ * the graph, another one with softmax outputs predicts the placement): no message passing,
+ * no sets. Reading taken (the paper gives no formula): the aggregate is the sum over ALL
+ * nodes of a per-node network, squashed as the pooling summaries of Sec. 2.2 step 3 are,
+ *     a = h( sum_{u in V} l(x_u) ),   logits = head(a),   probs = softmax(logits);
+ * the current node is in the sum like every other node and is told apart by its
+ * is-current feature alone. (The other ablation, the "simple partitioner", needs no entry
+ * point: it is placeto_policy_logits on embeddings of zero.)
+ *   w      : l: F -> d, h: d -> d, head: d -> hidden -> m (one or two layers each).
+ *   X      : DEVICE float[n][B][F] as built by placeto_build_features.
+ *   logits : DEVICE float[B][m] (out); probs: DEVICE float[B][m] (out) or NULL.
+ * One launch, no workspace; sums run in a fixed order (reproducible).
+ */
+typedef struct {
+    int32_t d, F, m;
+    placeto_mlp l, h, head;
+} placeto_aggregator_weights;
+placeto_status placeto_simple_aggregator(const placeto_graph *g, const placeto_aggregator_weights *w,
+                                         const float *X, int32_t B, float *logits, float *probs, void *stream);
+
+/*
  * What the kernels of the most recent call on `g` reported, read back after `stream` has
  * drained (this call synchronises it). The library's kernels never wait without a limit: a
  * wait on an asynchronous copy or on another warp that runs out makes the kernel leave, turn

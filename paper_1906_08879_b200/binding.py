@@ -32,6 +32,7 @@ EXPORTS = (
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
     "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulator_workspace_bytes", "placeto_simulate_runtime",
     "placeto_policy_gradient", "placeto_last_launch_count", "placeto_last_status", "placeto_debug_wait_timeout",
+    "placeto_simple_aggregator",
 )
 
 
@@ -53,6 +54,11 @@ class _Weights(ctypes.Structure):
     _fields_ = [("d", ctypes.c_int32), ("F", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("f_down", _Mlp), ("g_down", _Mlp), ("f_up", _Mlp), ("g_up", _Mlp),
                 ("l", _Mlp * 3), ("h", _Mlp * 3), ("head", _Mlp)]
+
+
+class _AggWeights(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("F", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("l", _Mlp), ("h", _Mlp), ("head", _Mlp)]
 
 
 class _LevelView(ctypes.Structure):
@@ -80,7 +86,7 @@ def _load() -> ctypes.CDLL:
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
                  "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime", "placeto_policy_gradient",
-                 "placeto_last_status", "placeto_debug_wait_timeout"):
+                 "placeto_last_status", "placeto_debug_wait_timeout", "placeto_simple_aggregator"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -405,6 +411,31 @@ def placeto_policy_gradient(g: Graph, w: Weights, X, H_down, H_up, cur, actions,
                                         _stream(stream)),
            "placeto_policy_gradient")
     return grads
+
+
+class AggregatorWeights:
+    """Device copies of the simple aggregator's three networks ({"d", "F", "m", "l", "h", "head"})."""
+
+    def __init__(self, weights: dict, device="cuda"):
+        self.d, self.F, self.m = int(weights["d"]), int(weights["F"]), int(weights["m"])
+        self._w = Weights({"d": self.d, "F": self.F, "m": self.m}, device)
+        self.c = _AggWeights()
+        self.c.d, self.c.F, self.c.m = self.d, self.F, self.m
+        dev = torch.device(device)
+        for name in ("l", "h", "head"):
+            setattr(self.c, name, self._w._mlp(weights[name], dev))
+
+
+def placeto_simple_aggregator(g: Graph, w: AggregatorWeights, X, logits=None, probs=None, stream=None):
+    """The "simple aggregator" ablation: softmax(head(h(sum over all nodes of l(x_u))))."""
+    B = X.shape[1]
+    if logits is None:
+        logits = torch.empty((B, w.m), dtype=torch.float32, device=X.device)
+    if probs is None:
+        probs = torch.empty((B, w.m), dtype=torch.float32, device=X.device)
+    _check(_lib.placeto_simple_aggregator(g.handle, ctypes.byref(w.c), _p(X), ctypes.c_int32(B), _p(logits),
+                                          _p(probs), _stream(stream)), "placeto_simple_aggregator")
+    return logits, probs
 
 
 def placeto_last_status(g: Graph, ws=None, stream=None) -> int:

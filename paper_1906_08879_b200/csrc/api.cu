@@ -844,6 +844,24 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
                                               static_cast<cudaStream_t>(stream)));
 }
 
+placeto_status placeto_simple_aggregator(const placeto_graph *g, const placeto_aggregator_weights *w,
+                                         const float *X, int32_t B, float *logits, float *probs, void *stream) {
+    t_launches = 0;
+    if (!g || !g->on_device || !w || B < 1 || !on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
+    g->calls.fetch_add(1);
+    if (w->d < 1 || w->F < 1 || w->m < 1) return PLACETO_ERR_INVALID_ARG;
+    if (w->d > PLACETO_MAX_D || w->F > PLACETO_MAX_F || w->m > PLACETO_MAX_M + 4) return PLACETO_ERR_UNSUPPORTED;
+    if (!mlp_ok(w->l, w->F, w->d) || !mlp_ok(w->h, w->d, w->d) || !mlp_ok(w->head, w->d, w->m))
+        return PLACETO_ERR_INVALID_ARG;
+    if ((size_t)B * g->host.n > (size_t)1 << 31) return PLACETO_ERR_UNSUPPORTED;
+    if (!X || !logits || !aligned16(X) || !aligned16(logits) || (probs && !aligned16(probs)))
+        return PLACETO_ERR_INVALID_ARG;
+    const cudaError_t e = launch_simple_aggregator(to_dev(w->l), to_dev(w->h), to_dev(w->head), X, g->host.n, B, w->F,
+                                                   w->d, w->m, logits, probs, g->info,
+                                                   static_cast<cudaStream_t>(stream));
+    return e == cudaErrorNotSupported ? PLACETO_ERR_UNSUPPORTED : cuda_status(e);
+}
+
 placeto_status placeto_last_status(const placeto_graph *g, const void *workspace, void *stream) {
     if (!g || !g->on_device) return PLACETO_ERR_INVALID_ARG;
     const char *at = static_cast<const char *>(workspace);

@@ -285,6 +285,11 @@ cudaError_t launch_embed_tc(const EmbedArgs &a, const DeviceInfo &di, cudaStream
 // time-out path without faulting or hanging anything.
 cudaError_t launch_wait_timeout_probe(const StatusSlot &status, cudaStream_t stream);
 
+// aggregator.cu: the "simple aggregator" policy (no message passing, no sets), one block per state
+cudaError_t launch_simple_aggregator(const DevMlp &l, const DevMlp &h, const DevMlp &head, const float *X, int n,
+                                     int B, int F, int d, int m, float *logits, float *probs, const DeviceInfo &di,
+                                     cudaStream_t stream);
+
 // policy_generic.cu: pooling partial sums, then per-state finalisation + head + softmax.
 int pool_chunks(int n, int B, const DeviceInfo &di);
 cudaError_t launch_policy_generic(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream);
