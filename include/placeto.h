@@ -312,7 +312,7 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
  * Readings where the paper is silent: one run time per operation whatever the
  * device; a tensor is sent once to each distinct device that hosts a child; a free
  * device or bus starts the head of its queue at once; equal time stamps are handled
- * in the order the events were created; peak memory is not modelled.
+ * in the order the events were created.
  *
  * cost, bytes : DEVICE float[n].          dev : DEVICE uint8[P][n], devices < m.
  * bandwidth   : > 0, in units of bytes[] per unit of cost[].
@@ -325,6 +325,30 @@ placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cos
                                         const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
                                         double *runtime, void *workspace, size_t workspace_bytes,
                                         void *stream);
+
+/*
+ * The same simulation with the devices' peak memory and the memory-penalised run time
+ * (Appendix A.5: the operations' start and end time stamps together with the tensor sizes
+ * predict the peak memory utilisation of the devices; Appendix A.7: R(p) = r if m <= M,
+ * r + c (m - M) otherwise, m the largest peak over the devices, M the memory limit, c a
+ * scale factor, 2 in the paper's experiments).
+ * Reading taken for the release of tensors, which the paper leaves open: a copy of an
+ * operation's output occupies the producer's device from the START of the producer until
+ * every child placed there has finished and every transfer of it to another device is done;
+ * it occupies another device from the START of the transfer there until every child placed
+ * there has finished; the output of an operation without children is never released.
+ *
+ * mem_limit, mem_scale : M and c, in the units of bytes[] and of cost[] per unit of bytes[].
+ * runtime     : DEVICE double[P] or NULL.       peak_memory : DEVICE double[P][m] or NULL.
+ * penalised   : DEVICE double[P] or NULL, R(p). At least one of the three must be given.
+ * Everything else as for placeto_simulate_runtime (same workspace size, NaN for a
+ * placement that names a device >= m, bit-reproducible sums).
+ */
+placeto_status placeto_simulate_placements(const placeto_graph *g, const float *cost, const float *bytes,
+                                           const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
+                                           double mem_limit, double mem_scale, double *runtime,
+                                           double *peak_memory, double *penalised, void *workspace,
+                                           size_t workspace_bytes, void *stream);
 
 /*
  * Gradient of the training objective with respect to every weight and bias of the

@@ -32,7 +32,7 @@ EXPORTS = (
     "placeto_policy_forward", "placeto_policy_forward_host", "placeto_policy_logits_static",
     "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulator_workspace_bytes", "placeto_simulate_runtime",
     "placeto_policy_gradient", "placeto_last_launch_count", "placeto_last_status", "placeto_debug_wait_timeout",
-    "placeto_simple_aggregator",
+    "placeto_simple_aggregator", "placeto_simulate_placements",
 )
 
 
@@ -86,7 +86,8 @@ def _load() -> ctypes.CDLL:
                  "placeto_build_features", "placeto_embed_forward", "placeto_policy_logits",
                  "placeto_policy_forward", "placeto_policy_forward_host",
                  "placeto_policy_logits_static", "placeto_episode_rollout", "placeto_embed_rounds", "placeto_simulate_runtime", "placeto_policy_gradient",
-                 "placeto_last_status", "placeto_debug_wait_timeout", "placeto_simple_aggregator"):
+                 "placeto_last_status", "placeto_debug_wait_timeout", "placeto_simple_aggregator",
+                 "placeto_simulate_placements"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -379,6 +380,27 @@ def placeto_simulate_runtime(g: Graph, cost, nbytes, dev, m: int, bandwidth: flo
                                          _p(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
            "placeto_simulate_runtime")
     return runtime
+
+
+def placeto_simulate_placements(g: Graph, cost, nbytes, dev, m: int, bandwidth: float, mem_limit: float,
+                                mem_scale: float, ws=None, stream=None):
+    """Run time [P], peak memory per device [P][m] and memory-penalised run time R(p) [P]
+    (float64) of the P placements in `dev` (uint8 [P][n])."""
+    P = dev.shape[0]
+    runtime = torch.empty((P,), dtype=torch.float64, device=dev.device)
+    peak = torch.empty((P, m), dtype=torch.float64, device=dev.device)
+    pen = torch.empty((P,), dtype=torch.float64, device=dev.device)
+    if ws is None:
+        need = int(_lib.placeto_simulator_workspace_bytes(g.handle, ctypes.c_int32(P), ctypes.c_int32(m)))
+        if need == 0:
+            raise PlacetoError(1, "placeto_simulator_workspace_bytes")
+        ws = torch.empty(need, dtype=torch.uint8, device=dev.device)
+    _check(_lib.placeto_simulate_placements(g.handle, _p(cost), _p(nbytes), _p(dev), ctypes.c_int32(P),
+                                            ctypes.c_int32(m), ctypes.c_double(bandwidth), ctypes.c_double(mem_limit),
+                                            ctypes.c_double(mem_scale), _p(runtime), _p(peak), _p(pen), _p(ws),
+                                            ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "placeto_simulate_placements")
+    return runtime, peak, pen
 
 
 def zero_gradients(weights: dict, device="cuda") -> "Weights":

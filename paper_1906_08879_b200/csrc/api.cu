@@ -756,28 +756,42 @@ size_t placeto_simulator_workspace_bytes(const placeto_graph *g, int32_t P, int3
     return sim_workspace_bytes(g->host.n, (int)g->host.n_edges, m, P);
 }
 
-placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cost, const float *bytes,
-                                        const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
-                                        double *runtime, void *workspace, size_t workspace_bytes,
-                                        void *stream) {
+placeto_status placeto_simulate_placements(const placeto_graph *g, const float *cost, const float *bytes,
+                                           const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
+                                           double mem_limit, double mem_scale, double *runtime,
+                                           double *peak_memory, double *penalised, void *workspace,
+                                           size_t workspace_bytes, void *stream) {
     t_launches = 0;
     if (!g || !g->on_device || P < 1 || m < 1 || m > PLACETO_MAX_M) return PLACETO_ERR_INVALID_ARG;
-    if (!(bandwidth > 0.0) || !on_graph_device(g)) return PLACETO_ERR_INVALID_ARG;
+    if (!(bandwidth > 0.0) || !(mem_scale >= 0.0) || mem_limit != mem_limit || !on_graph_device(g))
+        return PLACETO_ERR_INVALID_ARG;
     g->calls.fetch_add(1);
-    if (!cost || !bytes || !dev || !runtime || !workspace) return PLACETO_ERR_INVALID_ARG;
-    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(runtime) ||
-        !aligned16(workspace))
+    if (!cost || !bytes || !dev || !workspace || (!runtime && !peak_memory && !penalised)) return PLACETO_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(bytes) || !aligned16(dev) || !aligned16(workspace) ||
+        (runtime && !aligned16(runtime)) || (peak_memory && !aligned16(peak_memory)) ||
+        (penalised && !aligned16(penalised)))
         return PLACETO_ERR_INVALID_ARG;
     if (workspace_bytes < sim_workspace_bytes(g->host.n, (int)g->host.n_edges, m, P))
         return PLACETO_ERR_WORKSPACE;
     SimArgs a;
     a.n = g->host.n; a.n_edges = (int)g->host.n_edges; a.m = m; a.P = P;
     a.child_ptr = g->d_child_ptr; a.child = g->d_child; a.n_parents = g->d_n_parents;
+    a.parent_ptr = g->d_parent_ptr; a.parent = g->d_parent;
     a.cost = cost; a.bytes = bytes; a.dev = dev;
     a.bandwidth = bandwidth;
-    a.runtime = runtime;
+    a.mem_limit = mem_limit; a.mem_scale = mem_scale;
+    a.runtime = runtime; a.peak_memory = peak_memory; a.penalised = penalised;
     a.workspace = static_cast<char *>(workspace);
     return cuda_status(launch_simulator(a, static_cast<cudaStream_t>(stream)));
+}
+
+placeto_status placeto_simulate_runtime(const placeto_graph *g, const float *cost, const float *bytes,
+                                        const uint8_t *dev, int32_t P, int32_t m, double bandwidth,
+                                        double *runtime, void *workspace, size_t workspace_bytes,
+                                        void *stream) {
+    if (!runtime) return PLACETO_ERR_INVALID_ARG;
+    return placeto_simulate_placements(g, cost, bytes, dev, P, m, bandwidth, 0.0, 0.0, runtime, nullptr, nullptr,
+                                       workspace, workspace_bytes, stream);
 }
 
 placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_weights *w, const float *X,

@@ -113,10 +113,14 @@ struct EpisodeArgs {
 struct SimArgs {
     int n, n_edges, m, P;
     const int *child_ptr, *child, *n_parents;   // by node id
+    const int *parent_ptr, *parent;             // by node id, ascending
     const float *cost, *bytes;                  // [n]
     const uint8_t *dev;                         // [P][n]
     double bandwidth;
-    double *runtime;                            // [P]
+    double mem_limit, mem_scale;                // M and c of the memory-penalised run time
+    double *runtime;                            // [P] or null
+    double *peak_memory;                        // [P][m] or null
+    double *penalised;                          // [P] or null
     char *workspace;
 };
 

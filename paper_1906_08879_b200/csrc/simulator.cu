@@ -20,6 +20,17 @@
 // sent once to each distinct device hosting a child; a free device or bus starts
 // the head of its queue in the handler that filled it (a Wakeup with the current
 // time stamp); operations without parents are queued in ascending id at time 0.
+//
+// Peak memory (Appendix A.5: the operations' start and end time stamps together
+// with the tensor sizes predict the devices' peak memory; when a tensor is
+// released is left open). Reading: a copy of an output tensor occupies the
+// producer's device from the start of the producer until every child there has
+// finished and every transfer of it is done; it occupies another device from
+// the start of the transfer there until every child there has finished; outputs
+// without children are never released. The memory-penalised run time of
+// Appendix A.7 is R(p) = r if m <= M, r + c (m - M) otherwise, m the largest
+// peak over the devices. Byte counts are doubles added and subtracted in event
+// order (parents in ascending id inside an event): reproducible bit for bit.
 #include <cfloat>
 
 #include "kernels.cuh"
@@ -34,7 +45,7 @@ constexpr int kMaxM = PLACETO_MAX_M;
 // per placement: ints  pending[n], op_next[n], tr_op[T], tr_dst[T], tr_next[T], sent_mark[m * ?]
 // with T = min(n_edges, n * (m - 1)) transfer records at most
 __host__ __device__ inline size_t sim_ints(int n, int n_edges) {
-    return 2 * (size_t)n + 3 * (size_t)n_edges;
+    return 3 * (size_t)n + 3 * (size_t)n_edges;     // + tr_left[n]: transfers of a tensor not yet done
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -45,7 +56,8 @@ simulate_kernel(const SimArgs a) {
     int *base = reinterpret_cast<int *>(a.workspace);
     auto at = [&](size_t i) -> int & { return base[i * P + p]; };
     const size_t o_pending = 0, o_next = n, o_trop = 2 * (size_t)n, o_trdst = o_trop + a.n_edges,
-                 o_trnext = o_trdst + a.n_edges;
+                 o_trnext = o_trdst + a.n_edges, o_trleft = o_trnext + a.n_edges;
+    constexpr int kFinished = -1;            // value of pending[] once the operation has run
     const uint8_t *dev = a.dev + (size_t)p * n;
 
     // small per-device state in local memory
@@ -54,11 +66,28 @@ simulate_kernel(const SimArgs a) {
     int op_seq[kMaxM], tr_seq[kMaxM];
     double op_end[kMaxM], tr_end[kMaxM];
     int sent[kMaxM];                          // last operation whose output was queued for the device
+    double mem[kMaxM], peak[kMaxM];           // bytes held now / at most
     for (int d = 0; d < m; ++d) {
         q_head[d] = q_tail[d] = t_head[d] = t_tail[d] = -1;
         run_op[d] = run_tr[d] = -1;
         sent[d] = -1;
+        mem[d] = peak[d] = 0.0;
     }
+    auto hold = [&](int d, int o) {
+        mem[d] += (double)a.bytes[o];
+        if (mem[d] > peak[d]) peak[d] = mem[d];
+    };
+    // the copy of u's output on device d goes once no child there and no transfer needs it
+    auto maybe_release = [&](int u, int d) {
+        const int e0 = a.child_ptr[u], e1 = a.child_ptr[u + 1];
+        if (e0 == e1) return;
+        for (int e = e0; e < e1; ++e) {
+            const int c = a.child[e];
+            if (dev[c] == d && at(o_pending + c) != kFinished) return;
+        }
+        if (d == dev[u] && at(o_trleft + u) > 0) return;
+        mem[d] -= (double)a.bytes[u];
+    };
     int seq = 0, n_tr = 0, done = 0;
     double last = 0.0;
 
@@ -72,6 +101,7 @@ simulate_kernel(const SimArgs a) {
         q_head[d] = at(o_next + v);
         if (q_head[d] < 0) q_tail[d] = -1;
         run_op[d] = v;
+        hold(d, v);
         op_end[d] = now + (double)a.cost[v];
         op_seq[d] = seq++;
     };
@@ -80,12 +110,14 @@ simulate_kernel(const SimArgs a) {
         t_head[d] = at(o_trnext + r);
         if (t_head[d] < 0) t_tail[d] = -1;
         run_tr[d] = r;
+        hold(at(o_trdst + r), at(o_trop + r));
         tr_end[d] = now + (double)a.bytes[at(o_trop + r)] / a.bandwidth;
         tr_seq[d] = seq++;
     };
 
     for (int v = 0; v < n; ++v) {
         at(o_pending + v) = a.n_parents[v];
+        at(o_trleft + v) = 0;
         if (a.n_parents[v] == 0 && dev[v] < m) push_op(dev[v], v);
     }
     for (int d = 0; d < m; ++d)
@@ -111,6 +143,9 @@ simulate_kernel(const SimArgs a) {
             run_op[d] = -1;
             ++done;
             last = now;
+            at(o_pending + o) = kFinished;
+            for (int e = a.parent_ptr[o]; e < a.parent_ptr[o + 1]; ++e)      // the inputs o read here
+                if (dev[a.parent[e]] < m) maybe_release(a.parent[e], d);
             for (int e = a.child_ptr[o]; e < a.child_ptr[o + 1]; ++e) {
                 const int c = a.child[e], dc = dev[c];
                 if (dc >= m) continue;
@@ -121,6 +156,7 @@ simulate_kernel(const SimArgs a) {
                         at(o_trop + r) = o;
                         at(o_trdst + r) = dc;
                         at(o_trnext + r) = -1;
+                        at(o_trleft + o) += 1;
                         if (t_tail[d] < 0) t_head[d] = r; else at(o_trnext + t_tail[d]) = r;
                         t_tail[d] = r;
                     }
@@ -134,6 +170,8 @@ simulate_kernel(const SimArgs a) {
             const int d = who, r = run_tr[d];
             run_tr[d] = -1;
             const int o = at(o_trop + r), to = at(o_trdst + r);
+            at(o_trleft + o) -= 1;
+            maybe_release(o, d);
             for (int e = a.child_ptr[o]; e < a.child_ptr[o + 1]; ++e) {
                 const int c = a.child[e];
                 if (dev[c] == to && --at(o_pending + c) == 0) push_op(to, c);
@@ -143,7 +181,15 @@ simulate_kernel(const SimArgs a) {
         }
     }
     // a device id outside [0, m) leaves operations unplaced: report NaN
-    a.runtime[p] = done == n ? last : __longlong_as_double(0x7ff8000000000000LL);
+    const double nan = __longlong_as_double(0x7ff8000000000000LL);
+    const bool ok = done == n;
+    if (a.runtime) a.runtime[p] = ok ? last : nan;
+    double top = 0.0;
+    for (int d = 0; d < m; ++d) {
+        if (a.peak_memory) a.peak_memory[(size_t)p * m + d] = ok ? peak[d] : nan;
+        top = peak[d] > top ? peak[d] : top;
+    }
+    if (a.penalised) a.penalised[p] = !ok ? nan : (top <= a.mem_limit ? last : last + a.mem_scale * (top - a.mem_limit));
 }
 
 }  // namespace

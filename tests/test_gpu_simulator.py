@@ -93,3 +93,57 @@ def test_errors_and_invalid_devices():
     with pytest.raises(placeto.PlacetoError) as e:
         placeto.placeto_simulate_runtime(g, dev_t(cost), dev_t(size), dev_t(devs.astype(np.uint8)), m, 0.0)
     assert e.value.status == 1
+
+
+def test_peak_memory_and_penalised_runtime_bit_exact():
+    """placeto_simulate_placements against the CPU simulator: run time, per-device peak
+    memory and R(p) (Appendix A.5, A.7) are doubles produced by the same operations in the
+    same order."""
+    for seed in range(4):
+        r = rng(90 + seed)
+        n = int(r.integers(5, 60))
+        m = int(r.integers(1, 7))
+        src, dst = random_dag(r, n, float(r.uniform(0.05, 0.4)))
+        cost = r.lognormal(0, 1, n).astype(np.float32)
+        size = r.lognormal(3, 1.5, n).astype(np.float32)
+        devs = r.integers(0, m, size=(41, n))
+        bw = float(r.uniform(1, 50))
+        limit = float(np.percentile(size, 90)) * 2
+        g = placeto.Graph(n, src, dst)
+        rt, peak, pen = placeto.placeto_simulate_placements(g, dev_t(cost), dev_t(size), dev_t(devs.astype(np.uint8)),
+                                                            m, bw, limit, 2.0)
+        torch.cuda.synchronize()
+        want_rt, want_peak, want_pen = simulator.placements(n, src, dst, cost, size, devs, m, bw, limit, 2.0)
+        np.testing.assert_array_equal(rt.cpu().numpy(), want_rt)
+        np.testing.assert_array_equal(peak.cpu().numpy(), want_peak)
+        np.testing.assert_array_equal(pen.cpu().numpy(), want_pen)
+        assert (pen.cpu().numpy() >= rt.cpu().numpy()).all() and (pen.cpu().numpy() > rt.cpu().numpy()).any()
+
+
+def test_memory_timelines_by_hand_on_the_gpu():
+    src = np.array([0, 0, 1], np.int32); dst = np.array([1, 2, 3], np.int32)
+    cost = np.ones(4, np.float32); size = np.array([10, 20, 5, 50], np.float32)
+    devs = np.array([[0, 0, 1, 0], [0, 0, 0, 0]], np.uint8)
+    g = placeto.Graph(4, src, dst)
+    rt, peak, pen = placeto.placeto_simulate_placements(g, dev_t(cost), dev_t(size), dev_t(devs), 2, 0.1, 75.0, 2.0)
+    torch.cuda.synchronize()
+    assert rt.cpu().tolist() == [102.0, 4.0]
+    assert peak.cpu().tolist() == [[80.0, 15.0], [75.0, 0.0]]
+    assert pen.cpu().tolist() == [102.0 + 2.0 * 5.0, 4.0]
+
+
+def test_workload_graph_memory():
+    cfg = configs.make("inception", B=1)
+    r = rng(11)
+    n, m = cfg["n"], cfg["m"]
+    devs = r.integers(0, m, size=(64, n))
+    g = placeto.Graph(n, cfg["src"], cfg["dst"])
+    rt, peak, pen = placeto.placeto_simulate_placements(g, dev_t(cfg["cost"]), dev_t(cfg["bytes"]),
+                                                        dev_t(devs.astype(np.uint8)), m, 1e4, 1e6, 2.0)
+    torch.cuda.synchronize()
+    sel = np.arange(0, 64, 8)
+    want_rt, want_peak, want_pen = simulator.placements(n, cfg["src"], cfg["dst"], cfg["cost"], cfg["bytes"],
+                                                        devs[sel], m, 1e4, 1e6, 2.0)
+    np.testing.assert_array_equal(rt.cpu().numpy()[sel], want_rt)
+    np.testing.assert_array_equal(peak.cpu().numpy()[sel], want_peak)
+    np.testing.assert_array_equal(pen.cpu().numpy()[sel], want_pen)

@@ -1,5 +1,5 @@
 """Pins of the CPU runtime simulator (oracle/simulator.py) against timelines
-that the execution model of the paper's Appendix A.4 fixes by hand: one device,
+that the execution model of the paper's Appendix A.5 fixes by hand: one device,
 chains, independent chains, a fork-join with a transfer in each direction, a
 bus that serialises two transfers, FIFO order on a device, and bounds and
 closed forms on random graphs (critical path, device load, exact scaling).
@@ -115,3 +115,108 @@ def test_bounds_and_closed_forms_on_random_graphs(seed):
     assert t2 == 2 * t
     # a faster link never makes a chain-free schedule of one device slower
     assert simulator.runtime(n, src, dst, cost, size, np.zeros(n, int), m, 1.0) == pytest.approx(c64.sum())
+
+
+# ------------------------------------------------ peak memory and R(p) ----
+
+def _sim(src, dst, cost, size, dev, m, bw=1.0):
+    n = len(cost)
+    return simulator.simulate(n, np.asarray(src), np.asarray(dst), np.asarray(cost, np.float32),
+                              np.asarray(size, np.float32), dev, m, bw)
+
+
+def test_memory_timelines_by_hand():
+    """Appendix A.5: start and end of every operation plus the tensor sizes give
+    the devices' peak memory. Timelines small enough to follow by eye."""
+    # chain a -> b -> c on one device, sizes 10, 20, 5:
+    # a runs: 10; b runs: 10 + 20 = 30; b done frees a's output: 20; c runs: 25; c done frees b's: 5
+    r, peak = _sim([0, 1], [1, 2], [1, 1, 1], [10, 20, 5], [0, 0, 0], 1)
+    assert r == 3.0 and peak.tolist() == [30.0]
+    # a on device 0 feeds b on device 1: the receive buffer counts from the start of the transfer
+    # device 0: 10 while a runs and until its output has left; device 1: 10, then 10 + 20 while b runs
+    r, peak = _sim([0], [1], [1, 1], [10, 20], [0, 1], 2, bw=10.0)
+    assert r == 3.0 and peak.tolist() == [10.0, 30.0]
+    # fork a -> {b, c} on one device: a's output stays until BOTH children are done
+    # a: 10; b: 30; b done: a still needed by c; c: 35; c done frees a's
+    r, peak = _sim([0, 0], [1, 2], [1, 1, 1], [10, 20, 5], [0, 0, 0], 1)
+    assert peak.tolist() == [35.0]
+    # the same fork with c on device 1: device 0 holds a's output until b is done AND the copy has left
+    # device 0: a 10, b +20 = 30; device 1: copy of a 10, c +5 = 15
+    r, peak = _sim([0, 0], [1, 2], [1, 1, 1], [10, 20, 5], [0, 0, 1], 2, bw=10.0)
+    assert peak.tolist() == [30.0, 15.0]
+    # a -> {b on device 0, c on device 1}, b -> e on device 0, a slow link (the copy of a's output
+    # is under way from t = 1 to t = 101): a's output stays at home while it is being sent, so e
+    # runs on top of it. device 0: a 10, b 30, e 30 + 50 = 80; device 1: copy 10, c 15
+    r, peak = _sim([0, 0, 1], [1, 2, 3], [1, 1, 1, 1], [10, 20, 5, 50], [0, 0, 1, 0], 2, bw=0.1)
+    assert r == 102.0 and peak.tolist() == [80.0, 15.0]
+    # outputs of operations without children are never released: three roots on one device pile up
+    r, peak = _sim([], [], [1, 1, 1], [4, 5, 6], [0, 0, 0], 1)
+    assert peak.tolist() == [15.0]
+
+
+def test_memory_invariants_on_random_graphs():
+    r = rng(77)
+    for _ in range(6):
+        n, m = 25, 3
+        src, dst = random_dag(r, n, 0.15)
+        cost = r.lognormal(0, 1, n).astype(np.float32)
+        size = r.integers(1, 50, n).astype(np.float32)      # integers: sums are exact
+        dev = r.integers(0, m, n)
+        _, peak = simulator.simulate(n, src, dst, cost, size, dev, m, 7.0)
+        chi, _ = simulator.children_lists(n, src, dst)
+        for d in range(m):
+            own = [v for v in range(n) if dev[v] == d]
+            # a device holds at least its largest own output and all its childless outputs at the end
+            if own:
+                assert peak[d] >= max(size[v] for v in own)
+                assert peak[d] >= sum(size[v] for v in own if not chi[v])
+            # and never more than everything that is ever placed or copied there
+            copies = sum(size[u] for u in range(n) if dev[u] != d and any(dev[c] == d for c in chi[u]))
+            assert peak[d] <= sum(size[v] for v in own) + copies
+        # one device, no transfers: the peak does not depend on the bandwidth
+        a = simulator.simulate(n, src, dst, cost, size, np.zeros(n, int), 1, 1.0)[1]
+        b = simulator.simulate(n, src, dst, cost, size, np.zeros(n, int), 1, 99.0)[1]
+        assert a.tolist() == b.tolist()
+
+
+def test_memory_penalised_runtime():
+    """Appendix A.7: R(p) = r below the limit, r + c (m - M) above it."""
+    assert simulator.penalised_runtime(3.0, 10.0, 10.7, 2.0) == 3.0
+    assert simulator.penalised_runtime(3.0, 10.7, 10.7, 2.0) == 3.0
+    assert simulator.penalised_runtime(3.0, 12.7, 10.7, 2.0) == 3.0 + 2.0 * 2.0
+    src, dst = np.array([0, 0]), np.array([1, 2])
+    devs = np.array([[0, 0, 0], [0, 0, 1]])
+    r, peaks, pen = simulator.placements(3, src, dst, np.ones(3, np.float32), np.array([10, 20, 5], np.float32),
+                                         devs, 2, 10.0, 32.0, 2.0)
+    assert peaks.tolist() == [[35.0, 0.0], [30.0, 15.0]]
+    assert pen[0] == r[0] + 2.0 * 3.0 and pen[1] == r[1]
+
+
+@pytest.mark.parametrize("old,new", [
+    ("        if any(dev[c] == d and not finished[c] for c in chi[u]):\n            return\n", ""),   # freed at the first child
+    ("        hold(to, o)\n", ""),                                                                  # receive buffer not counted
+    ("        if d == dev[u] and tr_left[u] > 0:\n            return\n", ""),                      # freed before it was sent
+    ("return r if peak <= mem_limit else r + scale * (peak - mem_limit)",
+     "return r if peak <= mem_limit else r - scale * (peak - mem_limit)"),                          # penalty sign
+], ids=["freed at first child", "receive buffer dropped", "freed before sent", "penalty sign"])
+def test_planted_memory_mistakes_are_caught(old, new, monkeypatch):
+    import importlib.util, os, sys, tempfile
+    path = simulator.__file__
+    source = open(path).read()
+    assert source.count(old) == 1
+    with tempfile.TemporaryDirectory() as tmp:
+        mut = os.path.join(tmp, "mutant_simulator.py")
+        open(mut, "w").write(source.replace(old, new))
+        spec = importlib.util.spec_from_file_location("mutant_simulator", mut)
+        module = importlib.util.module_from_spec(spec)
+        spec.loader.exec_module(module)
+    this = sys.modules[__name__]
+    monkeypatch.setattr(this, "simulator", module)
+    caught = False
+    for pin in (test_memory_timelines_by_hand, test_memory_penalised_runtime, test_memory_invariants_on_random_graphs):
+        try:
+            pin()
+        except AssertionError:
+            caught = True
+            break
+    assert caught
