@@ -372,8 +372,10 @@ placeto_status placeto_simulate_placements(const placeto_graph *g, const float *
  *                   set of states can then be differentiated in several calls).
  * workspace       : DEVICE, at least placeto_workspace_bytes(.., PLACETO_CALL_GRADIENT, 0):
  *                   about 2 * n * B * (2 * (hidden_f + hidden_g) + 6 d) + 3 n B d floats.
- * Shapes: two-layer ReLU f and g, single-layer ReLU l_i and h_i, two-layer head with a
- * ReLU hidden layer and a linear output; otherwise PLACETO_ERR_UNSUPPORTED.
+ * Shapes: ReLU f and g of one layer (the paper's own, Appendix A.7) or two, single-layer
+ * ReLU l_i and h_i, two-layer head with a ReLU hidden layer and a linear output; otherwise
+ * PLACETO_ERR_UNSUPPORTED. A single-layer f or g is differentiated as the two-layer network
+ * relu(I relu(W x + b) + 0) that it equals bit for bit.
  */
 #define PLACETO_GRAD_ACCUMULATE 1u
 placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_weights *w, const float *X,

@@ -83,6 +83,7 @@ placeto_status pool_weights_ok(const placeto_weights *w) {
 struct Layout {
     size_t status;                 // 256 bytes at the start: the status word of the call
     size_t msg[2], msg_alt[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
+    size_t grad, grad_extra;       // gradient call: its intermediates; identity layers of single-layer f, g
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
     int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
 };
@@ -103,10 +104,15 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         L.msg[1] = take(n * B * d * sizeof(float));
     }
     if (call == PLACETO_CALL_GRADIENT) {
-        const int Hf = std::max(w->f_down.hidden_dim, w->f_up.hidden_dim);
-        const int Hg = std::max(w->g_down.hidden_dim, w->g_up.hidden_dim);
-        L.total = policy_gradient_workspace_floats((int)n, B, w->d, w->F, w->m, Hf, Hg, w->head.hidden_dim) *
-                  sizeof(float);
+        // a single-layer network is differentiated as the two-layer network it equals (see
+        // placeto_policy_gradient): its hidden width is then its output width
+        auto hidden = [](const placeto_mlp &net) { return net.n_layers == 2 ? net.hidden_dim : net.out_dim; };
+        const int Hf = std::max(hidden(w->f_down), hidden(w->f_up));
+        const int Hg = std::max(hidden(w->g_down), hidden(w->g_up));
+        L.grad = take(policy_gradient_workspace_floats((int)n, B, w->d, w->F, w->m, Hf, Hg, w->head.hidden_dim) *
+                      sizeof(float));
+        L.grad_extra = take(4 * 2 * (d * d + d) * sizeof(float));
+        L.total = off;
         return L;
     }
     if (call == PLACETO_CALL_EMBED_ROUNDS) {
@@ -831,6 +837,8 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
         !aligned16(actions) || !aligned16(advantages))
         return PLACETO_ERR_INVALID_ARG;
     GradArgs a{};
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     a.n = g->host.n; a.B = B; a.d = w->d; a.F = w->F; a.m = w->m;
     a.relation = g->d_relation;
     a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
@@ -840,6 +848,25 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
     a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
     for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
     a.head = to_dev(w->head);
+    // The paper's own f and g are single layers (Appendix A.7). y = relu(W x + b) is, bit for
+    // bit, the two-layer network relu(I relu(W x + b) + 0): the second ReLU sees values >= 0.
+    // The kernels differentiate that form; its identity layer lives in the workspace and the
+    // gradient of the identity is written to scratch beside it and dropped.
+    float *extra = reinterpret_cast<float *>(ws + L.grad_extra);
+    const size_t dd = (size_t)w->d * w->d, one = dd + w->d;
+    DevMlp *mp[4] = {&a.f[0], &a.f[1], &a.g[0], &a.g[1]};
+    bool widened[4] = {false, false, false, false};
+    for (int k = 0; k < 4; ++k) {
+        DevMlp &net = *mp[k];
+        if (net.n_layers != 1 || net.act != 0 || net.final_act != 1) continue;
+        float *eye = extra + (size_t)k * 2 * one;
+        if (launch_identity_layer(eye, w->d, st) != cudaSuccess) return PLACETO_ERR_CUDA;
+        net.n_layers = 2;
+        net.hidden_dim = net.out_dim;
+        net.W2 = eye;
+        net.b2 = eye + dd;
+        widened[k] = true;
+    }
     if (!policy_gradient_applicable(a)) return PLACETO_ERR_UNSUPPORTED;
     a.X = X; a.H[0] = H_down; a.H[1] = H_up;
     a.cur = cur; a.actions = actions; a.advantages = advantages; a.beta = beta;
@@ -854,8 +881,13 @@ placeto_status placeto_policy_gradient(const placeto_graph *g, const placeto_wei
     a.gg[0] = out(grads->g_down); a.gg[1] = out(grads->g_up);
     for (int i = 0; i < 3; ++i) { a.gl[i] = out(grads->l[i]); a.gh[i] = out(grads->h[i]); }
     a.ghead = out(grads->head);
-    return cuda_status(launch_policy_gradient(a, g->info, static_cast<float *>(workspace),
-                                              static_cast<cudaStream_t>(stream)));
+    GradOut *gp[4] = {&a.gf[0], &a.gf[1], &a.gg[0], &a.gg[1]};
+    for (int k = 0; k < 4; ++k)
+        if (widened[k]) {
+            gp[k]->W2 = extra + (size_t)k * 2 * one + one;
+            gp[k]->b2 = gp[k]->W2 + dd;
+        }
+    return cuda_status(launch_policy_gradient(a, g->info, reinterpret_cast<float *>(ws + L.grad), st));
 }
 
 placeto_status placeto_simple_aggregator(const placeto_graph *g, const placeto_aggregator_weights *w,

@@ -566,6 +566,19 @@ cudaError_t weight_grads(const WeightJobs &jobs, cudaStream_t stream) {
 
 }  // namespace
 
+namespace {
+__global__ void identity_layer_kernel(float *dst, int d) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < d * d + d) dst[i] = (i < d * d && i / d == i % d) ? 1.f : 0.f;
+}
+}  // namespace
+
+cudaError_t launch_identity_layer(float *dst, int d, cudaStream_t stream) {
+    identity_layer_kernel<<<(d * d + d + 255) / 256, 256, 0, stream>>>(dst, d);
+    count_launch();
+    return cudaGetLastError();
+}
+
 bool policy_gradient_applicable(const GradArgs &a) {
     auto relu2 = [](const DevMlp &m) { return m.n_layers == 2 && m.act == 0 && m.final_act == 1; };
     auto relu1 = [](const DevMlp &m) { return m.n_layers == 1 && m.act == 0 && m.final_act == 1; };

@@ -245,6 +245,9 @@ bool policy_gradient_applicable(const GradArgs &a);
 size_t policy_gradient_workspace_floats(int n, int B, int d, int F, int m, int Hf, int Hg, int Hh);
 cudaError_t launch_policy_gradient(GradArgs a, const DeviceInfo &di, float *ws, cudaStream_t stream);
 
+// writes the d x d identity matrix followed by d zeros (an identity layer: W2 = I, b2 = 0)
+cudaError_t launch_identity_layer(float *dst, int d, cudaStream_t stream);
+
 // embed_generic.cu: dimension-generic message passing. schedule is one of
 // PLACETO_PER_LEVEL / PLACETO_SLICED / PLACETO_COOPERATIVE.
 cudaError_t launch_embed_generic(const EmbedArgs &a, const DeviceInfo &di, unsigned schedule,

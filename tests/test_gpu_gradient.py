@@ -115,9 +115,19 @@ def test_reproducible_and_unsupported_shapes():
     b = gpu_gradient(cfg, actions, adv, 0.1)
     for key, t in a.tensors.items():
         assert torch.equal(t, b.tensors[key]), key
-    # single-layer f and g (the paper's Appendix A.7 shapes) are not differentiated
+    # identity activations are not differentiated
     r = rng(6)
-    cfg["weights"] = states.policy_weights(r, 32, 8, 4, 1, 0, 0.2)
+    cfg["weights"] = states.policy_weights(r, 32, 8, 4, 2, 1, 0.2)
     with pytest.raises(placeto.PlacetoError) as e:
         gpu_gradient(cfg, actions, adv, 0.0)
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("d,m", [(8, 3), (32, 4)])
+def test_single_layer_networks_as_in_the_paper(d, m):
+    """Appendix A.7: f and g are single layers. Every gradient array against the checker."""
+    cfg, actions, adv = small_case(21 + d, n=15, m=m, d=d, B=19)
+    r = rng(d)
+    cfg["weights"] = states.policy_weights(r, d, m + 4, m, 1, 0, 0.2)
+    grads = gpu_gradient(cfg, actions, adv, 0.05)
+    compare(cfg, grads, gradient.gradient(cfg, actions, adv, 0.05))
