@@ -86,6 +86,7 @@ struct Layout {
     size_t grad, grad_extra;       // gradient call: its intermediates; identity layers of single-layer f, g
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
     int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
+    int chunks_tc, chunk_nodes_tc; // and of the d = 64 tensor-core kernel (0 when it cannot apply)
 };
 
 // Workspace layout shared by every call; a call uses the leading part it needs.
@@ -124,9 +125,10 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
     if (w->F >= 4 && w->F <= 16 && (w->F & 3) == 0) {
         if (w->d == 32) pool_d32_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
         if (w->d == 64) pool_d64_chunks((int)n, B, w->F, g->info, &L.chunk_nodes32, &L.chunks32);
+        if (w->d == 64) pool_tc_chunks((int)n, B, g->info, &L.chunk_nodes_tc, &L.chunks_tc);
     }
     if (call == PLACETO_CALL_LOGITS || (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE))
-        L.partial = take((size_t)std::max(L.chunks, L.chunks32) * B * 3 * d * sizeof(float));
+        L.partial = take((size_t)std::max(L.chunks, std::max(L.chunks32, L.chunks_tc)) * B * 3 * d * sizeof(float));
     if (call >= PLACETO_CALL_FORWARD && call <= PLACETO_CALL_EPISODE) {
         L.X = take(n * B * F * sizeof(float));
         L.H[0] = take(n * B * d * sizeof(float));
@@ -242,6 +244,12 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     a.logits = logits; a.probs = probs;
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d; a.m = w->m;
     const bool fast32 = pool_d32_applicable(a), fast64 = pool_d64_applicable(a);
+    if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) && L.chunks_tc > 0 && pool_tc_applicable(a)) {
+        a.chunks = L.chunks_tc; a.chunk_nodes = L.chunk_nodes_tc;
+        cudaError_t e = launch_pool_tc(a, g->info, stream, after_own_kernel);
+        if (e == cudaSuccess) return cuda_status(launch_pool_head(a, g->info, stream));
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     if (!(flags & PLACETO_GENERIC) && L.chunks32 > 0 && (fast32 || fast64)) {
         a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
         cudaError_t e = fast32 ? launch_pool_d32(a, g->info, stream, after_own_kernel)

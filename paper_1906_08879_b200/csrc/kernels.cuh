@@ -315,4 +315,10 @@ void pool_d64_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes
 cudaError_t launch_pool_d64(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
                             bool overlap = false);
 
+// policy_tc.cu: the same partial sums for d = 64 on tcgen05 tensor cores (weights of the current
+// set in tensor memory, two operand tiles in shared memory, accumulators in tensor memory)
+bool pool_tc_applicable(const PoolArgs &a);
+void pool_tc_chunks(int n, int B, const DeviceInfo &di, int *chunk_nodes, int *chunks);
+cudaError_t launch_pool_tc(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap = false);
+
 }  // namespace placeto
