@@ -84,6 +84,7 @@ struct Layout {
     size_t status;                 // 256 bytes at the start: the status word of the call
     size_t msg[2], msg_alt[2], partial, X, H[2], cost, bytes, dev, placed, cur, logits, probs, total;
     size_t grad, grad_extra;       // gradient call: its intermediates; identity layers of single-layer f, g
+    size_t compact;                // episode call: the compact states [n][E]
     int chunks, chunk_nodes;       // node chunks of the generic pooling kernel
     int chunks32, chunk_nodes32;   // and of the d = 32 / d = 64 kernel (0 when neither can apply)
     int chunks_tc, chunk_nodes_tc; // and of the d = 64 tensor-core kernel (0 when it cannot apply)
@@ -144,6 +145,7 @@ Layout make_layout(const placeto_graph *g, const placeto_weights *w, int B, plac
         L.probs = take((size_t)B * m * sizeof(float));
     }
     if (call == PLACETO_CALL_EPISODE) {
+        L.compact = take(n * B);
         L.placed = take(n * B);
         L.cur = take((size_t)B * sizeof(int32_t));
         L.logits = take((size_t)B * m * sizeof(float));
@@ -195,9 +197,11 @@ placeto_status cuda_status(cudaError_t e) {
 
 placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const float *X, int B,
                          float *H_down, float *H_up, char *ws, const Layout &L, uint32_t flags,
-                         cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false) {
+                         cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false,
+                         const CompactState *compact = nullptr) {
     EmbedArgs a;
     a.status = status;
+    a.compact = compact ? *compact : CompactState{};
     a.lv[0] = g->lv[0]; a.lv[1] = g->lv[1];
     a.f[0] = to_dev(w->f_down); a.f[1] = to_dev(w->f_up);
     a.g[0] = to_dev(w->g_down); a.g[1] = to_dev(w->g_up);
@@ -208,6 +212,8 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d;
     a.max_level_width = g->host.max_level_width;
     const unsigned schedule = pick_schedule(flags);
+    if (compact != nullptr)      // only the d = 32 kernel builds features from compact states
+        return cuda_status(launch_embed_d32(a, g->info, stream, after_own_kernel));
     if ((flags & PLACETO_TCGEN05) && !(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) &&
         schedule == PLACETO_SLICED && embed_tc_applicable(a)) {
         cudaError_t e = launch_embed_tc(a, g->info, stream, after_own_kernel);
@@ -232,9 +238,12 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
 placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const float *X,
                         const float *H_down, const float *H_up, const int32_t *cur, int B,
                         float *logits, float *probs, char *ws, const Layout &L, uint32_t flags,
-                        cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false) {
+                        cudaStream_t stream, const StatusSlot &status, bool after_own_kernel = false,
+                        const CompactState *compact = nullptr, const EpisodeStep *step = nullptr) {
     PoolArgs a;
     a.status = status;
+    a.compact = compact ? *compact : CompactState{};
+    a.step = step ? *step : EpisodeStep{};
     for (int i = 0; i < 3; ++i) { a.l[i] = to_dev(w->l[i]); a.h[i] = to_dev(w->h[i]); }
     a.head = to_dev(w->head);
     a.X = X; a.H[0] = H_down; a.H[1] = H_up;
@@ -244,6 +253,11 @@ placeto_status run_pool(const placeto_graph *g, const placeto_weights *w, const 
     a.logits = logits; a.probs = probs;
     a.n = g->host.n; a.B = B; a.F = w->F; a.d = w->d; a.m = w->m;
     const bool fast32 = pool_d32_applicable(a), fast64 = pool_d64_applicable(a);
+    if (compact != nullptr) {    // only the d = 32 kernel and the fast head kernel take compact states
+        a.chunks = L.chunks32; a.chunk_nodes = L.chunk_nodes32;
+        cudaError_t e = launch_pool_d32(a, g->info, stream, after_own_kernel);
+        return cuda_status(e == cudaSuccess ? launch_pool_head(a, g->info, stream) : e);
+    }
     if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) && L.chunks_tc > 0 && pool_tc_applicable(a)) {
         a.chunks = L.chunks_tc; a.chunk_nodes = L.chunk_nodes_tc;
         cudaError_t e = launch_pool_tc(a, g->info, stream, after_own_kernel);
@@ -751,6 +765,48 @@ placeto_status placeto_episode_rollout(const placeto_graph *g, const placeto_wei
     float *probs = reinterpret_cast<float *>(ws + L.probs);
     ep.X = X;
     const StatusSlot status = new_status_slot(g, ws, L);
+
+    // Where every kernel of a step takes compact states (the d = 32 sweep and pooling kernels
+    // and the fast head kernel), the episodes run without a feature tensor: one byte per (node,
+    // episode) is the whole state, and the head kernel makes the transition itself.
+    bool compact_path = false;
+    if (!(flags & (PLACETO_GENERIC | PLACETO_TENSOR | PLACETO_PER_LEVEL | PLACETO_COOPERATIVE)) && w->m < 63 &&
+        L.chunks32 > 0) {
+        EmbedArgs ea;
+        ea.lv[0] = g->lv[0]; ea.lv[1] = g->lv[1];
+        ea.f[0] = to_dev(w->f_down); ea.f[1] = to_dev(w->f_up);
+        ea.g[0] = to_dev(w->g_down); ea.g[1] = to_dev(w->g_up);
+        ea.n = g->host.n; ea.B = E; ea.F = w->F; ea.d = w->d;
+        ea.max_level_width = g->host.max_level_width;
+        PoolArgs pa;
+        for (int i = 0; i < 3; ++i) { pa.l[i] = to_dev(w->l[i]); pa.h[i] = to_dev(w->h[i]); }
+        pa.head = to_dev(w->head);
+        pa.n = g->host.n; pa.B = E; pa.F = w->F; pa.d = w->d; pa.m = w->m;
+        pa.chunks = L.chunks32; pa.chunk_nodes = L.chunk_nodes32;
+        compact_path = embed_d32_fits(ea, g->info) && pool_d32_fits(pa, g->info) && pool_head_takes_compact(pa);
+    }
+    if (compact_path) {
+        CompactState cs;
+        cs.cost = cost; cs.bytes = bytes; cs.m = w->m;
+        uint8_t *state = reinterpret_cast<uint8_t *>(ws + L.compact);
+        cs.state = state;
+        cs.cur = ep.cur;
+        s = cuda_status(launch_episode_begin_compact(ep.n, E, order, dev, state, ep.cur, st));
+        EpisodeStep step;
+        step.enabled = 1; step.n = ep.n;
+        step.order = order; step.uniforms = uniforms;
+        step.state = state; step.cur = ep.cur;
+        step.logp = logp; step.actions = actions;
+        for (int t = 0; s == PLACETO_OK && t < ep.n; ++t) {
+            step.t = t;
+            s = run_embed(g, w, nullptr, E, Hd, Hu, ws, L, flags, st, status, true, &cs);
+            if (s == PLACETO_OK)
+                s = run_pool(g, w, nullptr, Hd, Hu, ep.cur, E, const_cast<float *>(ep.logits), probs, ws, L, flags, st,
+                             status, true, &cs, &step);
+        }
+        if (s == PLACETO_OK) s = cuda_status(launch_episode_end_compact(ep.n, E, state, dev, st));
+        return s;
+    }
     s = cuda_status(launch_episode_begin(ep, st));
     // the features of the initial states; every later step patches them in place
     if (s == PLACETO_OK)

@@ -175,7 +175,7 @@ after_g1:
         if (r == 0 || last_live) msg[((slot * S) + st[r]) * kD + lane] = fmaxf(acc[r], 0.f);
 }
 
-template <int F4>   // feature width padded to 4 * F4
+template <int F4, bool kCompact>   // feature width padded to 4 * F4; features built from compact states
 __global__ void __launch_bounds__(kThreads, 1)
 embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
     constexpr int KF = kD + 4 * F4;      // padded input width of f's first layer
@@ -252,6 +252,14 @@ embed_d32_kernel(const EmbedArgs a, const D32Plan p) {
         if (warp != kWarps - 1) return;
         const int q0 = level_ptr[level], width = level_ptr[level + 1] - q0;
         float *dst = xstage + (size_t)(level & 1) * p.x_floats;
+        if (kCompact) {
+            // no X tensor: the level's features from one byte per (node, state)
+            for (int i = lane; i < width * nb; i += 32) {       // one (node, state) pair per lane
+                const int q = nb == 1 ? i : (int)__umulhi((unsigned)i, magic_nb), s = i - q * nb;
+                compact_features(a.compact, meta[q0 + q].w, b_first + s, (int)B, dst + (size_t)i * F);
+            }
+            return;
+        }
         for (int i = lane; i < width * per; i += 32) {
             const int q = per == 1 ? i : (int)__umulhi((unsigned)i, magic_per);
             const int piece = i - q * per;
@@ -309,8 +317,9 @@ bool embed_d32_applicable(const EmbedArgs &a) {
     return true;
 }
 
-cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
-                             bool overlap) {
+namespace {
+// slice size and shared-memory layout; false when not even one state per block fits
+bool plan_d32(const EmbedArgs &a, const DeviceInfo &di, D32Plan *out) {
     D32Plan p;
     const int target = std::max(1, di.sm_count / 2);            // blocks per direction
     const int want = std::max(1, std::min(a.B, target));
@@ -319,7 +328,7 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
     const int KF = kD + 4 * F4;
     const size_t budget = (size_t)std::min(di.max_smem_optin, 227 * 1024) - 1024;
     const int max_slots = std::max(a.lv[0].n_slots, a.lv[1].n_slots);
-    if (max_slots >= 0xffff) return cudaErrorNotSupported;   // slot ids are packed into 16 bits
+    if (max_slots >= 0xffff) return false;   // slot ids are packed into 16 bits
     size_t ints = 0;
     for (int dir = 0; dir < 2; ++dir) {
         const DevLevels &lv = a.lv[dir];
@@ -333,16 +342,32 @@ cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
     };
     // narrower slices when the shared memory does not fit (more blocks: they queue up)
     while (p.S > 1 && need(p.S) > budget) --p.S;
-    if (need(p.S) > budget) return cudaErrorNotSupported;
+    if (need(p.S) > budget) return false;
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.x_floats = x_floats(p.S);
     p.smem_bytes = need(p.S);
+    *out = p;
+    return true;
+}
+}  // namespace
+
+bool embed_d32_fits(const EmbedArgs &a, const DeviceInfo &di) {
+    D32Plan p;
+    return embed_d32_applicable(a) && plan_d32(a, di, &p);
+}
+
+cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
+                             bool overlap) {
+    D32Plan p;
+    if (!plan_d32(a, di, &p)) return cudaErrorNotSupported;
+    const int F4 = (a.F + 3) / 4;
     void (*kern)(const EmbedArgs, const D32Plan) = nullptr;
+    const bool compact = a.compact.state != nullptr;
     switch (F4) {
-        case 1: kern = embed_d32_kernel<1>; break;
-        case 2: kern = embed_d32_kernel<2>; break;
-        case 3: kern = embed_d32_kernel<3>; break;
-        case 4: kern = embed_d32_kernel<4>; break;
+        case 1: kern = compact ? embed_d32_kernel<1, true> : embed_d32_kernel<1, false>; break;
+        case 2: kern = compact ? embed_d32_kernel<2, true> : embed_d32_kernel<2, false>; break;
+        case 3: kern = compact ? embed_d32_kernel<3, true> : embed_d32_kernel<3, false>; break;
+        case 4: kern = compact ? embed_d32_kernel<4, true> : embed_d32_kernel<4, false>; break;
         default: return cudaErrorNotSupported;
     }
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,

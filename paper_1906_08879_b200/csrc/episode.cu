@@ -4,11 +4,17 @@
 // sample driven by a caller-supplied uniform number), writes it into the
 // placement, marks the node visited, records the log-probability of the choice
 // and makes the next node of the visiting order current. With it a whole episode
-// runs as a stream of launches without a host round trip per step. A step changes
-// the raw features of two nodes only (the node just placed: device one-hot,
-// current flag off, visited flag on; the next node: current flag on), so the
-// same thread patches those rows of X in place and the feature tensor is built
-// once per episode, not once per step.
+// runs as a stream of launches without a host round trip per step.
+//
+// Two forms. Where the step's kernels take compact states (the d = 32 sweep and pooling
+// kernels with the fast head kernel), there is no feature tensor at all: the state of the
+// E episodes is one byte per (node, episode) plus the current node, the kernels build the
+// features on the fly, and the transition itself is the head kernel's last step (see
+// EpisodeStep); this file then only converts the placement to and from compact states.
+// Elsewhere the transition is the kernel below: a step changes the raw features of two
+// nodes only (the node just placed: device one-hot, current flag off, visited flag on; the
+// next node: current flag on), so the thread of an episode patches those rows of X in
+// place and the feature tensor is built once per episode, not once per step.
 #include <cmath>
 
 #include "kernels.cuh"
@@ -75,7 +81,51 @@ __global__ void episode_step_kernel(EpisodeArgs a, int t) {
     }
 }
 
+// compact states from the initial placement: state[v][e] = device (63 for an id that no device
+// carries: its one-hot is all zero), nothing visited; cur[e] = order[0]
+__global__ void episode_begin_compact_kernel(int n, int E, const int *__restrict__ order,
+                                             const uint8_t *__restrict__ dev, uint8_t *__restrict__ state,
+                                             int *__restrict__ cur) {
+    const size_t total = (size_t)E * n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t v = i / E, e = i - v * E;
+        const uint8_t d = dev[e * n + v];
+        state[i] = d < 63 ? d : 63;
+    }
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < E) cur[e] = order[0];
+}
+
+__global__ void episode_end_compact_kernel(int n, int E, const uint8_t *__restrict__ state,
+                                           uint8_t *__restrict__ dev) {
+    dependency_wait();
+    const size_t total = (size_t)E * n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t e = i / n, v = i - e * n;
+        // a node that was never visited keeps the device it came with (63 stood for any id >= 63)
+        const uint8_t s = state[v * E + e];
+        if (s & 0x80) dev[i] = s & 63;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_episode_begin_compact(int n, int E, const int *order, const uint8_t *dev, uint8_t *state,
+                                         int *cur, cudaStream_t stream) {
+    const int blocks = std::max(1, std::min(2048, (int)(((size_t)E * n + kThreads - 1) / kThreads)));
+    const int need = (E + kThreads - 1) / kThreads;       // every episode needs its thread
+    episode_begin_compact_kernel<<<std::max(blocks, need), kThreads, 0, stream>>>(n, E, order, dev, state, cur);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_episode_end_compact(int n, int E, const uint8_t *state, uint8_t *dev, cudaStream_t stream) {
+    const int blocks = std::max(1, std::min(2048, (int)(((size_t)E * n + kThreads - 1) / kThreads)));
+    cudaError_t err = launch_overlapped(true, episode_end_compact_kernel, dim3(blocks), dim3(kThreads), 0, stream,
+                                        n, E, state, dev);
+    count_launch();
+    return err;
+}
 
 cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream) {
     const int blocks = std::max(1, std::min(1024, (int)(((size_t)a.E * a.n + kThreads - 1) / kThreads)));

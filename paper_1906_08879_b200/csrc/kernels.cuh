@@ -75,6 +75,54 @@ __device__ __forceinline__ void report_status(const StatusSlot &s, int code) {
 #endif
 #endif
 
+// Compact placement states (Sec. 2.1): per (node, state) one byte - the node's device in
+// the low six bits, bit 7 set once the node has been visited - and the current node per
+// state. Together with the per-node cost and output size they determine every raw feature
+// (Sec. 2.2 step 1), so a kernel given them builds x on the fly instead of reading X:
+// one byte instead of 4 F per node and state.
+struct CompactState {
+    const float *cost, *bytes;   // [n]
+    const uint8_t *state;        // [n][B]; null: the features come from X
+    const int *cur;              // [B]
+    int m;
+};
+#ifdef __CUDACC__
+// feature k of node v in state b: [cost, bytes, one-hot_m(device), v == cur, visited]
+__device__ __forceinline__ float compact_feature(const CompactState &c, int v, int b, int B, int k) {
+    if (k == 0) return c.cost[v];
+    if (k == 1) return c.bytes[v];
+    const unsigned s = c.state[(size_t)v * B + b];
+    if (k < 2 + c.m) return (int)(s & 63u) == k - 2 ? 1.f : 0.f;
+    if (k == 2 + c.m) return c.cur[b] == v ? 1.f : 0.f;
+    return (float)(s >> 7);
+}
+// all F = m + 4 features of node v in state b into x[0 .. F): one state byte, the node's cost and
+// size, the state's current node
+__device__ __forceinline__ void compact_features(const CompactState &c, int v, int b, int B, float *x) {
+    const unsigned s = c.state[(size_t)v * B + b];
+    const int dev = (int)(s & 63u);
+    x[0] = c.cost[v];
+    x[1] = c.bytes[v];
+    for (int k = 0; k < c.m; ++k) x[2 + k] = k == dev ? 1.f : 0.f;
+    x[2 + c.m] = c.cur[b] == v ? 1.f : 0.f;
+    x[3 + c.m] = (float)(s >> 7);
+}
+#endif
+
+// The MDP transition fused into the head kernel (episodes on compact states): after the
+// logits of step t the thread of a state picks the device of the current node (argmax, or
+// the inverse CDF of the FP32 softmax at uniforms[e][t]), records it, marks the node visited
+// and makes order[t + 1] current.
+struct EpisodeStep {
+    int enabled, t, n;
+    const int *order;          // [n]
+    const float *uniforms;     // [E][n] or null (greedy)
+    uint8_t *state;            // [n][E] compact states, updated in place
+    int *cur;                  // [E], updated in place
+    float *logp;               // [E][n] by step, or null
+    uint8_t *actions;          // [E][n] by step, or null
+};
+
 struct EmbedArgs {
     DevLevels lv[2];
     DevMlp f[2], g[2];
@@ -84,6 +132,7 @@ struct EmbedArgs {
     int n, B, F, d;
     int max_level_width;   // widest level over both directions
     StatusSlot status;
+    CompactState compact;  // compact.state != null: X is not read
 };
 
 struct PoolArgs {
@@ -96,6 +145,8 @@ struct PoolArgs {
     int n, B, F, d, m;
     int chunks, chunk_nodes;
     StatusSlot status;
+    CompactState compact;  // compact.state != null: X is not read
+    EpisodeStep step;      // step.enabled: the head kernel also makes the MDP transition
 };
 
 struct EpisodeArgs {
@@ -235,6 +286,13 @@ cudaError_t launch_stage_inputs(const void *const (&src)[5], void *const (&dst)[
 // episode.cu: the MDP transition between two policy evaluations of an episode
 cudaError_t launch_episode_begin(const EpisodeArgs &a, cudaStream_t stream);
 cudaError_t launch_episode_step(const EpisodeArgs &a, int t, cudaStream_t stream);
+// compact states: state[v][e] from the initial placement dev[e][v] (nothing visited), cur[e] = order[0];
+// and back: dev[e][v] = the device of state[v][e]
+cudaError_t launch_episode_begin_compact(int n, int E, const int *order, const uint8_t *dev, uint8_t *state,
+                                         int *cur, cudaStream_t stream);
+cudaError_t launch_episode_end_compact(int n, int E, const uint8_t *state, uint8_t *dev, cudaStream_t stream);
+// true when an episode step on these shapes runs on kernels that take compact states
+bool pool_head_takes_compact(const PoolArgs &a);
 
 // simulator.cu: event-based run time of P placements, one thread each
 size_t sim_workspace_bytes(int n, int n_edges, int m, int P);
@@ -266,6 +324,7 @@ cudaError_t launch_embed_rounds_d32(const EmbedArgs &a, const DeviceInfo &di, in
 // networks of hidden width 32; returns cudaErrorNotSupported when the shapes or
 // the shared-memory budget do not fit (the caller then uses the generic kernel).
 bool embed_d32_applicable(const EmbedArgs &a);
+bool embed_d32_fits(const EmbedArgs &a, const DeviceInfo &di);   // applicable and within shared memory
 cudaError_t launch_embed_d32(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
                              bool overlap = false);
 
@@ -305,6 +364,7 @@ cudaError_t launch_pool_head(const PoolArgs &a, const DeviceInfo &di, cudaStream
 
 // policy_d32.cu: specialised partial sums for d = 32, F a multiple of 4, single-layer ReLU l_i
 bool pool_d32_applicable(const PoolArgs &a);
+bool pool_d32_fits(const PoolArgs &a, const DeviceInfo &di);      // applicable (a.chunk_nodes set) and within shared memory
 void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes, int *chunks);
 cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
                             bool overlap = false);

@@ -64,7 +64,7 @@ __device__ __forceinline__ void fma_rows(const pair_t *w, const float *const (&i
     }
 }
 
-template <int F4>
+template <int F4, bool kCompact>     // kCompact: the raw features come from compact states, not from X
 __global__ void __launch_bounds__(kThreads, 1)
 pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     constexpr int FP = 4 * F4;             // padded feature width
@@ -91,7 +91,7 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
     const unsigned h_bytes = (unsigned)(nb * kD * sizeof(float)), x_bytes = (unsigned)(nb * F * sizeof(float));
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
-        mbar_expect(&bar, 3 * w_bytes + (unsigned)nu * (2 * h_bytes + x_bytes));
+        mbar_expect(&bar, 3 * w_bytes + (unsigned)nu * (2 * h_bytes + (kCompact ? 0u : x_bytes)));
     }
     if (threadIdx.x < 3 * kD) bs[threadIdx.x] = a.l[threadIdx.x / kD].b1[threadIdx.x % kD];
     __syncthreads();
@@ -103,7 +103,15 @@ pool_d32_kernel(const PoolArgs a, const Pool32Plan p) {
         const size_t row = (size_t)(u0 + q) * B + b0;
         if (which == 0) bulk_load(hd + (size_t)q * kWarps * kD, a.H[0] + row * kD, h_bytes, &bar);
         else if (which == 1) bulk_load(hu + (size_t)q * kWarps * kD, a.H[1] + row * kD, h_bytes, &bar);
-        else bulk_load(xs + (size_t)q * kWarps * FP, a.X + row * F, x_bytes, &bar);
+        else if (!kCompact) bulk_load(xs + (size_t)q * kWarps * FP, a.X + row * F, x_bytes, &bar);
+    }
+    if (kCompact) {
+        // no X tensor: the tile's features from one byte per (node, state)
+        for (int i = threadIdx.x; i < nu * nb; i += kThreads) {     // one (node, state) pair per thread
+            const int q = i / nb, st = i - q * nb;
+            compact_features(a.compact, u0 + q, b0 + st, B, xs + (size_t)q * kWarps * FP + st * FP);
+        }
+        __syncthreads();
     }
     const bool landed = mbar_wait(&bar, 0);
     if (!landed && threadIdx.x == 0) report_status(a.status, PLACETO_ERR_TIMEOUT);
@@ -187,6 +195,12 @@ void pool_d32_chunks(int n, int B, int F, const DeviceInfo &di, int *chunk_nodes
     *chunks = (n + *chunk_nodes - 1) / *chunk_nodes;
 }
 
+bool pool_d32_fits(const PoolArgs &a, const DeviceInfo &di) {
+    const int E = 2 * kD + a.F;
+    const size_t bytes = ((size_t)(3 * E * kD + 3 * kD) + (size_t)a.chunk_nodes * kWarps * E) * sizeof(float);
+    return pool_d32_applicable(a) && a.chunk_nodes > 0 && bytes <= (size_t)di.max_smem_optin;
+}
+
 cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_t stream,
                             bool overlap) {
     Pool32Plan p;
@@ -197,10 +211,10 @@ cudaError_t launch_pool_d32(const PoolArgs &a, const DeviceInfo &di, cudaStream_
     if (p.smem_bytes > (size_t)di.max_smem_optin) return cudaErrorNotSupported;
     void (*kern)(const PoolArgs, const Pool32Plan) = nullptr;
     switch (a.F / 4) {
-        case 1: kern = pool_d32_kernel<1>; break;
-        case 2: kern = pool_d32_kernel<2>; break;
-        case 3: kern = pool_d32_kernel<3>; break;
-        case 4: kern = pool_d32_kernel<4>; break;
+        case 1: kern = a.compact.state ? pool_d32_kernel<1, true> : pool_d32_kernel<1, false>; break;
+        case 2: kern = a.compact.state ? pool_d32_kernel<2, true> : pool_d32_kernel<2, false>; break;
+        case 3: kern = a.compact.state ? pool_d32_kernel<3, true> : pool_d32_kernel<3, false>; break;
+        case 4: kern = a.compact.state ? pool_d32_kernel<4, true> : pool_d32_kernel<4, false>; break;
         default: return cudaErrorNotSupported;
     }
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,

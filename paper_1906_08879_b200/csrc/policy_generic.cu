@@ -405,7 +405,8 @@ pool_head_fast_kernel(const PoolArgs a) {
         if (c >= 0 && c < a.n)
             v = k < d ? a.H[0][((size_t)c * B + b) * d + k]
               : k < 2 * d ? a.H[1][((size_t)c * B + b) * d + (k - d)]
-                          : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
+              : a.compact.state != nullptr ? compact_feature(a.compact, c, b, B, k - 2 * d)
+                                           : a.X[((size_t)c * B + b) * F + (k - 2 * d)];
         zt[k * HS + s] = v;
     }
     __syncthreads();
@@ -524,6 +525,31 @@ pool_head_fast_kernel(const PoolArgs a) {
             a.logits[(size_t)b * m + k] = valid ? l[k] : nanf("");
             if (a.probs) a.probs[(size_t)b * m + k] = valid ? expf(l[k] - mx) / tot : nanf("");
         }
+        if (a.step.enabled) {
+            // The MDP transition of episode b (Sec. 2.1), fused here: greedy takes the largest
+            // logit (lowest index among equals), sampling the first k with p_0 + .. + p_k > u for
+            // p the FP32 softmax summed in index order (the last index if rounding leaves none).
+            const EpisodeStep &st = a.step;
+            int best = 0;
+            float top = l[0];
+            for (int k = 1; k < m; ++k)
+                if (l[k] > top) { top = l[k]; best = k; }
+            int action = best;
+            if (st.uniforms != nullptr) {
+                const float u = st.uniforms[(size_t)b * st.n + st.t];
+                float cum = 0.f;
+                action = m - 1;
+                for (int k = 0; k < m; ++k) {
+                    cum += expf(l[k] - mx) / tot;
+                    if (cum > u) { action = k; break; }
+                }
+            }
+            if (st.logp != nullptr) st.logp[(size_t)b * st.n + st.t] = (l[action] - mx) - logf(tot);
+            if (st.actions != nullptr) st.actions[(size_t)b * st.n + st.t] = (uint8_t)action;
+            const int v = st.order[st.t];
+            if (v >= 0 && v < st.n) st.state[(size_t)v * B + b] = (uint8_t)(action | 0x80);   // placed, visited
+            if (st.t + 1 < st.n) st.cur[b] = st.order[st.t + 1];
+        }
     }
 }
 
@@ -556,6 +582,8 @@ cudaError_t launch_head_fast(const PoolArgs &a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+bool pool_head_takes_compact(const PoolArgs &a) { return head_fast_applicable(a); }
 
 int pool_chunks(int n, int B, const DeviceInfo &di) {
     // enough (chunk, state-group) blocks to fill the device a few times over

@@ -79,13 +79,28 @@ def small_case(seed, n, m, d, E, p=0.2):
 
 
 @pytest.mark.parametrize("sampled", [False, True])
-@pytest.mark.parametrize("d,m", [(32, 4), (8, 3), (64, 8)])
-def test_small_graphs(d, m, sampled):
+@pytest.mark.parametrize("d,m,flags", [(32, 4, 0), (32, 4, placeto.PLACETO_TENSOR), (32, 3, 0), (8, 3, 0), (64, 8, 0)])
+def test_small_graphs(d, m, flags, sampled):
+    """d = 32 with F a multiple of 4 runs on compact states (one byte per node and episode, no
+    feature tensor, the transition inside the head kernel: three kernels per step); the other
+    cases, and d = 32 on the tensor kernel, keep the feature tensor and patch it (four)."""
     cfg, order, dev0, uni = small_case(100 * d + m, n=24, m=m, d=d, E=12)
     uniforms = uni if sampled else None
-    got = run_gpu(cfg, order, dev0, uniforms)
+    got = run_gpu(cfg, order, dev0, uniforms, flags)
     compare(cfg, order, dev0, uniforms, got, min_full=9)
-    assert got[3] >= 24 * 4 + 2          # three policy kernels and one transition per step
+    compact = d == 32 and m == 4 and flags == 0
+    assert got[3] == (24 * 3 + 2 if compact else 24 * 4 + 2)
+
+
+def test_compact_states_with_initial_devices_beyond_the_device_count():
+    """An initial placement may name devices the policy does not know (their one-hot is all
+    zero); nodes keep them until visited. E = 70 episodes: several per block in every kernel."""
+    cfg, order, dev0, uni = small_case(77, n=20, m=4, d=32, E=70)
+    dev0[:, ::3] = 200
+    dev0[:, 1::5] = 63
+    got = run_gpu(cfg, order, dev0, uni)
+    compare(cfg, order, dev0, uni, got, min_full=50)
+    assert got[3] == 20 * 3 + 2
 
 
 def test_reverse_order_and_single_episode():
