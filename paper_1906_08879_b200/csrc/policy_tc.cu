@@ -23,7 +23,7 @@
 //     per row: 256 + 256 + 4F contiguous bytes), split them and store them in
 //     the operand layout; a four-deep ring of tile descriptors (rows, flags,
 //     item) travels with the tiles; the node list of a (set, item) pair is compacted by all
-//     producer warps a pair ahead, and that pair's rows are pulled into L2 then;
+//     producer warps a pair ahead;
 //   - one thread issues the instructions of a tile into one of two accumulators
 //     and commits them to the barriers that free the tile and hand the
 //     accumulator over;
@@ -359,17 +359,6 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const PoolArgs a, 
             // the next pair's list, while the first tile's rows are on their way
             if (k + 1 < n_pairs) build_list(k + 1, lists[(k + 1) & 1], &cnt_next);
             asm volatile("bar.sync 1, %0;" ::"n"(kProdThreads) : "memory");   // next list complete
-            if (k + 1 < n_pairs) {
-                // pull the next pair's rows into L2 now, a whole pair ahead of their use
-                const int next_b = (first_item + ((k + 1) % my_items) * item_step) % B;
-                const int *next_list = lists[(k + 1) & 1];
-                for (int i = ptid; i < cnt_next * 5; i += kProdThreads) {
-                    const int r = i / 5, part = i - 5 * r;
-                    const size_t row = (size_t)next_list[r] * B + next_b;
-                    const float *at = part < 4 ? a.H[part >> 1] + row * kD + (part & 1) * 32 : a.X + row * F;
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(at));
-                }
-            }
             PT(0);
             const int n_tiles = max(1, (cnt + kTileRows - 1) / kTileRows);
             for (int t = 0; t < n_tiles; ++t) {
