@@ -108,10 +108,10 @@ def job_throughput(local_ms: float, states_per_rank: int, steps: int, dist=None,
     return states_per_rank * world * steps / (slowest * 1e-3), slowest
 
 
-def measured_traffic(workload: str):
+def measured_traffic(workload: str, flags: int = 0):
     """DRAM bytes per launch of the message-passing kernel from the committed ncu
-    summary of this workload (profiles/*.md), or None when there is none or the
-    kernel source has changed since the counters were taken."""
+    summary of this workload and these flags (profiles/*.md), or None when there is
+    none or the kernel source has changed since the counters were taken."""
     import glob
     import hashlib
     for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
@@ -121,6 +121,8 @@ def measured_traffic(workload: str):
                 k, _, v = line.partition(":")
                 fields[k.strip()] = v.strip()
         if fields.get("workload") != workload or "traffic_bytes_per_launch" not in fields:
+            continue
+        if int(fields.get("flags", "0")) != flags:
             continue
         src = os.path.join(ROOT, fields.get("kernel_source", ""))
         if not os.path.isfile(src):
@@ -482,7 +484,7 @@ def run_b200(args):
         hbm_src = "measured (MEASURED_PEAKS.json)"
     peak_tflops = sm_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
     achieved = flops_embed(cfg) * max(1, args.rounds) / (embed_ms * 1e-3) / 1e12
-    traffic, traffic_from = measured_traffic(cfg["name"])
+    traffic, traffic_from = measured_traffic(cfg["name"], args.flags)
     roofline = {"bound": "alu",
                 "kernel": ("message passing (embed_rounds, %d synchronous rounds, %d launches)" % (args.rounds, embed_launches)
                            if args.rounds > 0 else "message passing (embed_forward, %d launch(es))" % embed_launches),

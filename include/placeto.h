@@ -163,11 +163,16 @@ typedef struct {
 #define PLACETO_FMA_ONLY 16u   /* keep step 2 on the FP32 FMA pipes: do not use the tensor-core
                                   kernel (TF32 head + tail split, three products per step) that
                                   d = 64 otherwise takes */
-#define PLACETO_TENSOR 32u     /* use the tensor-core kernel of step 2 wherever it applies
-                                  (d = 32 or 64), also where the library would pick the FMA one */
+#define PLACETO_TENSOR 32u     /* use the tensor-core kernel of step 2 that gives every block whole 16-row
+                                  tiles (all warps on one layer at a time) wherever it applies (d = 32 or
+                                  64), also where the library would pick another one */
 #define PLACETO_TCGEN05 64u    /* d = 64: take the kernel built on tcgen05.mma with accumulators in tensor
                                   memory instead of the warp-level (mma.sync) tensor-core kernel that is
                                   the default there (measured slower at the configured batch sizes) */
+#define PLACETO_PIPELINE 128u  /* d = 64: take the kernel that runs the four layers of g and f as a pipeline
+                                  (a group of warps per layer, tiles of eight rows), also for batches so
+                                  large that the library would pick the 16-row-tile kernel (the default
+                                  up to eight states per thread block) */
 
 typedef enum {
     PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libplaceto_debug.so" if os.environ.get("PLACETO_
 
 # flags and enums of placeto.h
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8
-PLACETO_FMA_ONLY, PLACETO_TENSOR, PLACETO_TCGEN05 = 16, 32, 64
+PLACETO_FMA_ONLY, PLACETO_TENSOR, PLACETO_TCGEN05, PLACETO_PIPELINE = 16, 32, 64, 128
 PLACETO_GRAPH_DEVICE, PLACETO_GRAPH_HOST_ONLY = 0, 1
 CALL_EMBED, CALL_LOGITS, CALL_FORWARD, CALL_FORWARD_HOST, CALL_EPISODE, CALL_EMBED_ROUNDS, CALL_GRADIENT = 0, 1, 2, 3, 4, 5, 6
 

@@ -26,7 +26,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplaceto.so")
 LIB_DEBUG = os.path.join(HERE, "libplaceto_debug.so")
 
-SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "embed_d32.cu", "embed_d64.cu", "embed_mma.cu", "embed_tc.cu",
+SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "embed_d32.cu", "embed_d64.cu", "embed_mma.cu", "embed_pipe.cu", "embed_tc.cu",
            "policy_generic.cu", "policy_d32.cu", "policy_d64.cu", "episode.cu",
            "embed_rounds_d32.cu", "simulator.cu", "gradient.cu", "status.cu", "aggregator.cu", "policy_tc.cu"]
 

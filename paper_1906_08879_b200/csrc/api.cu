@@ -163,7 +163,7 @@ unsigned pick_schedule(unsigned flags) {
 
 bool flags_ok(uint32_t flags) {
     const uint32_t known = PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE |
-                           PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR | PLACETO_TCGEN05;
+                           PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR | PLACETO_TCGEN05 | PLACETO_PIPELINE;
     if (flags & ~known) return false;
     const uint32_t sched = flags & (PLACETO_PER_LEVEL | PLACETO_SLICED | PLACETO_COOPERATIVE);
     return (sched & (sched - 1)) == 0;   // at most one schedule
@@ -217,6 +217,12 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
     if ((flags & PLACETO_TCGEN05) && !(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY)) &&
         schedule == PLACETO_SLICED && embed_tc_applicable(a)) {
         cudaError_t e = launch_embed_tc(a, g->info, stream, after_own_kernel);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
+    // d = 64: the pipeline of layers where it is the faster one (or asked for), if it fits
+    if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR)) && schedule == PLACETO_SLICED &&
+        ((flags & PLACETO_PIPELINE) ? embed_pipe_applicable(a) : embed_pipe_preferred(a, g->info))) {
+        cudaError_t e = launch_embed_pipe(a, g->info, stream, after_own_kernel);
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
     const bool want_mma = (flags & PLACETO_TENSOR) ? embed_mma_applicable(a) : embed_mma_preferred(a);

@@ -340,6 +340,13 @@ bool embed_mma_preferred(const EmbedArgs &a);   // applicable and faster than th
 cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream,
                              bool overlap = false);
 
+// embed_pipe.cu: d = 64 as a pipeline of layers on mma.sync (a group of warps per layer of f and g,
+// tiles of eight rows handed from layer to layer through shared memory). cudaErrorNotSupported when
+// the schedule and the message slots do not fit in shared memory.
+bool embed_pipe_applicable(const EmbedArgs &a);
+bool embed_pipe_preferred(const EmbedArgs &a, const DeviceInfo &di);   // applicable and faster than the tile kernel
+cudaError_t launch_embed_pipe(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap = false);
+
 // embed_tc.cu: d = 64 on tcgen05 tensor cores with accumulators in tensor memory (TF32 head + tail
 // operands, all four partial products per instruction). A bounded wait that runs out inside the
 // kernel is reported through a.status as PLACETO_ERR_TIMEOUT.

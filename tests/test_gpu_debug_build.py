@@ -40,7 +40,7 @@ CHILD = textwrap.dedent('''
     # every specialised kernel on a case with several states per block: no index out of range
     cases = {}
     for d, m, flags in ((32, 4, 0), (32, 4, placeto.PLACETO_TENSOR), (64, 8, 0), (64, 8, placeto.PLACETO_FMA_ONLY),
-                        (64, 8, placeto.PLACETO_TCGEN05), (8, 2, 0)):
+                        (64, 8, placeto.PLACETO_TCGEN05), (64, 8, placeto.PLACETO_TENSOR), (8, 2, 0)):
         rng = np.random.Generator(np.random.PCG64(d + flags))
         n, src, dst = graphs.layered_dag(seed=5, levels=12, width=5)
         cfg = {"n": n, "src": src, "dst": dst, "m": m, "d": d, "F": m + 4, "B": 200}

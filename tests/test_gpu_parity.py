@@ -30,7 +30,7 @@ SCHEDULES = {"sliced": placeto.PLACETO_SLICED, "per_level": placeto.PLACETO_PER_
              "cooperative": placeto.PLACETO_COOPERATIVE,
              "generic_sliced": placeto.PLACETO_SLICED | placeto.PLACETO_GENERIC,
              "fma_only": placeto.PLACETO_FMA_ONLY, "tensor": placeto.PLACETO_TENSOR,
-             "tcgen05": placeto.PLACETO_TCGEN05}
+             "tcgen05": placeto.PLACETO_TCGEN05, "pipeline": placeto.PLACETO_PIPELINE}
 
 
 def dev_t(a):
@@ -125,7 +125,7 @@ def test_nmt(normalise, flags):
     compare(cfg, out, oracle.forward(cfg, threads=8))
 
 
-@pytest.mark.parametrize("flags", [0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TCGEN05])
+@pytest.mark.parametrize("flags", [0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR, placeto.PLACETO_TCGEN05])
 def test_nasnet_full_batch_sampled_states(flags):
     """Full size on the GPU (n ~ 2100, B = 512, d = 64); the checker evaluates
     a sample of states one by one (states are independent). At this batch the
@@ -213,7 +213,8 @@ def test_specialised_kernels_over_feature_widths(d, m):
     n = int(r.integers(30, 90))
     src, dst = random_dag(r, n, float(r.uniform(0.03, 0.12)))
     B = int(r.integers(3, 70))
-    for flags in (0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR, placeto.PLACETO_TCGEN05):
+    for flags in (0, placeto.PLACETO_FMA_ONLY, placeto.PLACETO_TENSOR, placeto.PLACETO_TCGEN05,
+                  placeto.PLACETO_PIPELINE):
         _small_case(n, src, dst, d=d, m=m, B=B, seed=m + d, schedule=flags)
 
 
@@ -224,6 +225,28 @@ def test_tcgen05_kernel_over_batch_sizes(B):
     r = rng(B)
     src, dst = random_dag(r, 60, 0.08)
     _small_case(60, src, dst, d=64, m=8, B=B, seed=B, schedule=placeto.PLACETO_TCGEN05)
+
+
+@pytest.mark.parametrize("B", [1, 7, 33, 300, 1200])
+def test_pipeline_kernel_over_batch_sizes(B):
+    """d = 64 as a pipeline of layers: one state per block (a tile holds rows of up to
+    eight nodes), a ragged last slice, and slices of up to 17 states, forced by the flag
+    (levels of more tiles than a ring holds, so tiles enter while others leave)."""
+    r = rng(B)
+    src, dst = random_dag(r, 60, 0.08)
+    _small_case(60, src, dst, d=64, m=8, B=B, seed=B, schedule=placeto.PLACETO_PIPELINE)
+
+
+def test_pipeline_kernel_on_a_deep_chain_and_a_wide_level():
+    n = 1500
+    src = list(range(n - 1)) + list(range(0, n - 40, 37))
+    dst = list(range(1, n)) + [i + 40 for i in range(0, n - 40, 37)]
+    _small_case(n, src, dst, d=64, m=8, B=10, seed=29, schedule=placeto.PLACETO_PIPELINE)
+    # 40 roots -> 12 nodes -> 1 sink with 20 states per block: levels of 100 and 30 tiles
+    r = rng(31)
+    src = list(range(40)) + [40 + i for i in range(12)]
+    dst = [40 + int(r.integers(0, 12)) for _ in range(40)] + [52] * 12
+    _small_case(53, src, dst, d=64, m=12, B=1480, seed=31, schedule=placeto.PLACETO_PIPELINE)
 
 
 def test_tcgen05_kernel_on_a_deep_chain_and_a_wide_level():
