@@ -15,9 +15,10 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# PLACETO_LIBRARY=debug selects the build whose kernels check their indices (build.py --debug)
-LIB_PATH = os.path.join(_HERE, "libplaceto_debug.so" if os.environ.get("PLACETO_LIBRARY") == "debug"
-                        else "libplaceto.so")
+# PLACETO_LIBRARY=debug selects the build whose kernels check their indices (build.py --debug),
+# PLACETO_LIBRARY=timers the one whose tcgen05 kernels print phase timers (build.py --timers)
+LIB_PATH = os.path.join(_HERE, {"debug": "libplaceto_debug.so", "timers": "libplaceto_timers.so"}.get(
+    os.environ.get("PLACETO_LIBRARY", ""), "libplaceto.so"))
 
 # flags and enums of placeto.h
 PLACETO_AUTO, PLACETO_PER_LEVEL, PLACETO_SLICED, PLACETO_COOPERATIVE, PLACETO_GENERIC = 0, 1, 2, 4, 8

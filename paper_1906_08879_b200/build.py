@@ -11,6 +11,12 @@ kernels check the schedule records, slot, node and state indices they stage and
 report a violation through the call's status record (see
 ``placeto_last_status``) instead of touching memory they should not. The
 binding loads it when the environment variable ``PLACETO_LIBRARY=debug`` is set.
+
+``build(timers=True)`` (``--timers``) makes ``libplaceto_timers.so`` with
+``-DPLACETO_PHASE_TIMERS``: the kernels built on tcgen05 (step 2 at d = 64 under
+PLACETO_TCGEN05, step 3 at d = 64) print, from block 0, the cycles each of their
+warp roles spent per phase. Selected with ``PLACETO_LIBRARY=timers``; a
+measuring aid, slower than the release build.
 """
 from __future__ import annotations
 
@@ -25,6 +31,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplaceto.so")
 LIB_DEBUG = os.path.join(HERE, "libplaceto_debug.so")
+LIB_TIMERS = os.path.join(HERE, "libplaceto_timers.so")
 
 SOURCES = ["api.cu", "plan.cpp", "features.cu", "embed_generic.cu", "embed_d32.cu", "embed_d64.cu", "embed_mma.cu", "embed_pipe.cu", "embed_tc.cu",
            "policy_generic.cu", "policy_d32.cu", "policy_d64.cu", "episode.cu",
@@ -49,14 +56,16 @@ def _stale(target: str, deps: list[str]) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False, timers: bool = False) -> str:
     """Compiles changed sources (in parallel) and links the library; returns its path."""
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(INCLUDE, "placeto.h"))
-    objdir = os.path.join(HERE, "_build", "debug" if debug else "release")
+    if debug and timers:
+        raise ValueError("one variant at a time")
+    objdir = os.path.join(HERE, "_build", "debug" if debug else "timers" if timers else "release")
     os.makedirs(objdir, exist_ok=True)
-    lib = LIB_DEBUG if debug else LIB
-    flags = NVCC_FLAGS + (["-DPLACETO_DEBUG"] if debug else [])
+    lib = LIB_DEBUG if debug else LIB_TIMERS if timers else LIB
+    flags = NVCC_FLAGS + (["-DPLACETO_DEBUG"] if debug else ["-DPLACETO_PHASE_TIMERS"] if timers else [])
     objs, jobs = [], []
     for src in SOURCES:
         path = os.path.join(CSRC, src)
@@ -81,4 +90,5 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv,
+                timers="--timers" in sys.argv))
