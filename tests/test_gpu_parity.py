@@ -237,6 +237,18 @@ def test_pipeline_kernel_over_batch_sizes(B):
     _small_case(60, src, dst, d=64, m=8, B=B, seed=B, schedule=placeto.PLACETO_PIPELINE)
 
 
+@pytest.mark.parametrize("B", [3, 40])
+def test_pipeline_kernel_on_degenerate_graphs(B):
+    """One node, no edges (one level of several tiles), chain, stars (fan-in 6: the gather's
+    neighbour loop), repeated edge, components: d = 64 through the pipeline of layers."""
+    s = placeto.PLACETO_PIPELINE
+    e = np.zeros(0, np.int32)
+    for n, src, dst in ((1, e, e), (5, e, e), (9, np.arange(8), np.arange(1, 9)),
+                        (7, np.zeros(6, np.int32), np.arange(1, 7)), (7, np.arange(1, 7), np.zeros(6, np.int32)),
+                        (4, [0, 0, 1, 2, 0], [1, 2, 3, 3, 1]), (7, [0, 1, 3, 4], [1, 2, 4, 5])):
+        _small_case(n, src, dst, d=64, m=4, B=B, seed=n + B, schedule=s)
+
+
 def test_pipeline_kernel_on_a_deep_chain_and_a_wide_level():
     n = 1500
     src = list(range(n - 1)) + list(range(0, n - 40, 37))
