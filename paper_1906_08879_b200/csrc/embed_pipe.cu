@@ -34,6 +34,7 @@
 #include <cuda_pipeline.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "kernels.cuh"
 
@@ -242,24 +243,11 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
     const float *X = a.X;
     float *__restrict__ H = a.H[dir];
 
-    // All sixteen warps run the same loop (one copy of the code in the instruction caches);
-    // what differs between the layers is data: the weights, where a tile is read and written,
-    // and a few steps under a condition that is uniform over the warp.
-    const DevMlp net = stage < 2 ? a.g[dir] : a.f[dir];
-    const bool second = stage & 1;
-    const bool wide = stage == 2;                    // f's first layer also reads the raw features
-    AFrag<NKF> w;
-    w.load(second ? net.W2 : net.W1, kD, wide ? kD + F : kD, c0, lane);
     const int col = c0 + g;                          // this lane finishes columns col and col + 8 of rows 2t, 2t + 1
-    const float b_lo = (second ? net.b2 : net.b1)[col], b_hi = (second ? net.b2 : net.b1)[col + 8];
-    const float *in_ring = stage == 0 ? ring0 : stage == 1 ? ring1 : stage == 2 ? ring2 : ring3;
-    float *out_ring = stage == 0 ? ring1 : stage == 1 ? ring2 : ring3;
-    const int in_P = stage == 2 ? PF : kP, out_P = stage == 1 ? PF : kP;
     // Hand-over: named barrier kFirstBar + ring * kRing + slot. There is no barrier for the way
     // back: the last layer's group, which also feeds the first ring, lets tile n + kRing in only
     // after it has taken tile n out of the last ring, so at most kRing tiles are between the
     // rings at any time and a slot is never rewritten before everybody has read it.
-    const int in_bar = kFirstBar + stage * kRing, out_bar = in_bar + kRing;
 
     // exact division of small non-negative numbers by a per-block constant
     const unsigned magic_nb = (unsigned)((0x100000000ull + nb - 1) / nb);
@@ -321,15 +309,30 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
         __pipeline_commit();
     };
 
+    // One copy of the walk per layer, so that what differs between the layers (which ring, the
+    // raw-feature columns, where h_v and m_u go, the gather) is decided at compile time.
+    auto walk = [&](auto stage_constant) {
+    constexpr int STAGE = decltype(stage_constant)::value;
+    constexpr bool second = STAGE & 1;
+    constexpr bool wide = STAGE == 2;                // f's first layer also reads the raw features
+    constexpr int NKW = wide ? NKF : NKD;
+    const DevMlp net = STAGE < 2 ? a.g[dir] : a.f[dir];
+    AFrag<NKW> w;
+    w.load(second ? net.W2 : net.W1, kD, wide ? kD + F : kD, c0, lane);
+    const float b_lo = (second ? net.b2 : net.b1)[col], b_hi = (second ? net.b2 : net.b1)[col + 8];
+    const float *in_ring = STAGE == 0 ? ring0 : STAGE == 1 ? ring1 : STAGE == 2 ? ring2 : ring3;
+    float *out_ring = STAGE == 0 ? ring1 : STAGE == 1 ? ring2 : ring3;
+    constexpr int in_P = STAGE == 2 ? PF : kP, out_P = STAGE == 1 ? PF : kP;
+    constexpr int in_bar = kFirstBar + STAGE * kRing, out_bar = in_bar + kRing;
     // The walk starts one level early, with nothing to compute: the last layer's group gathers
     // the first tiles of level 0 there and the second layer of g requests its raw features, in
     // the same code that does it between two levels (one call site each, inlined).
 #pragma unroll 1
     for (int level = -1; level < lv.n_levels; ++level) {
         const int p0 = level < 0 ? 0 : level_ptr[level], rows = level < 0 ? 0 : (level_ptr[level + 1] - p0) * nb;
-        const int n_tiles = level < 0 ? (stage == 3 ? 1 : 0) : (rows + kTile - 1) / kTile;
+        const int n_tiles = level < 0 ? (STAGE == 3 ? 1 : 0) : (rows + kTile - 1) / kTile;
         const float *xs = xstage + (size_t)(level & 1) * p.x_floats;
-        if (stage == 1) __pipeline_wait_prior(0);          // this level's raw features: requested a level ago
+        if (STAGE == 1) __pipeline_wait_prior(0);          // this level's raw features: requested a level ago
 #pragma unroll 1
         for (int j = 0; j < n_tiles; ++j) {
             if (level >= 0) {
@@ -343,11 +346,11 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                         if (r < rows) {
                             const int q = node_of_row(r);
                             const int4 m = meta[p0 + q];
-                            if (stage == 1) dst[i] = H + ((size_t)m.w * B + b_first + (r - q * nb)) * kD + col;
+                            if (STAGE == 1) dst[i] = H + ((size_t)m.w * B + b_first + (r - q * nb)) * kD + col;
                             else if (m.z >= 0) dst[i] = msg + ((size_t)m.z * S + (r - q * nb)) * kP + col;
                         }
                     }
-                    if (stage == 1 && x_mine) {
+                    if (STAGE == 1 && x_mine) {
                         // the raw features (zero padded) behind the d embedding columns of the output tile
                         const int r = kTile * j + x_row;
                         store_split(out_ring + slot * 2 * kTile * PF + x_row * PF + kD + x_col, kTile * PF,
@@ -356,10 +359,10 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 }
                 await_tile(in_bar + slot);
                 float c[4];
-                tile_product<NKF>(w, in_ring + slot * 2 * kTile * in_P, in_P, lane, wide, c);
+                tile_product<NKW>(w, in_ring + slot * 2 * kTile * in_P, in_P, lane, wide, c);
                 const float v[4] = {fmaxf(c[0] + b_lo, 0.f), fmaxf(c[1] + b_lo, 0.f), fmaxf(c[2] + b_hi, 0.f),
                                     fmaxf(c[3] + b_hi, 0.f)};      // (row 2t, col), (2t + 1, col), (2t, col + 8), (2t + 1, col + 8)
-                if (stage != 3) {
+                if (STAGE != 3) {
                     float *out = out_ring + slot * 2 * kTile * out_P + 2 * t * out_P + col;
                     const int tail = kTile * out_P;
                     store_split(out, tail, v[0]);
@@ -378,7 +381,7 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 }
                 ++tc;
             }
-            if (stage == 3) {
+            if (STAGE == 3) {
                 // Sums for the tiles ahead. Inside a level: one more tile for the one just taken
                 // (this level's messages go to slots that no row of this level reads). After the
                 // level's last tile: all its messages are written (group barrier), and the first
@@ -395,7 +398,14 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 for (; g_j < upto; ++g_j) gather(g_level, g_j);
             }
         }
-        if (stage == 1 && level + 1 < lv.n_levels) prefetch(level + 1);      // the other buffer: its level is done
+        if (STAGE == 1 && level + 1 < lv.n_levels) prefetch(level + 1);      // the other buffer: its level is done
+    }
+    };
+    switch (stage) {
+        case 0: walk(std::integral_constant<int, 0>{}); break;
+        case 1: walk(std::integral_constant<int, 1>{}); break;
+        case 2: walk(std::integral_constant<int, 2>{}); break;
+        default: walk(std::integral_constant<int, 3>{}); break;
     }
 }
 
