@@ -80,16 +80,20 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const unsigned (&a)[4], 
 }
 // Four 8 x 4 blocks of 32-bit words: lane i gives the address of row i % 8 of block i / 8 and
 // receives, from block j, word lane % 4 of row lane / 4 -- the B fragments of two k-steps.
-__device__ __forceinline__ void ldmatrix4(unsigned (&r)[4], const float *p) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+// `addr` is a shared-memory address, OFF a byte offset known at compile time (no address
+// arithmetic per instruction).
+template <int OFF>
+__device__ __forceinline__ void ldmatrix4(unsigned (&r)[4], unsigned addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4+%5];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(smem_addr(p))
+                 : "r"(addr), "n"(OFF)
                  : "memory");
 }
-__device__ __forceinline__ void ldmatrix2(unsigned (&r)[2], const float *p) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];"
+template <int OFF>
+__device__ __forceinline__ void ldmatrix2(unsigned (&r)[2], unsigned addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2+%3];"
                  : "=r"(r[0]), "=r"(r[1])
-                 : "r"(smem_addr(p))
+                 : "r"(addr), "n"(OFF)
                  : "memory");
 }
 // One warp's 16 columns [c0, c0 + 16) of a K x d matrix as A fragments of the transposed
@@ -112,58 +116,56 @@ struct AFrag {
     }
 };
 
-// c = (this warp's 16 columns of W)^T x (tile)^T for a tile of 8 rows in shared memory (heads at
-// `buf`, row stride P; tails kTile * P floats on), in the C-fragment layout
+// c = (this warp's 16 columns of W)^T x (tile)^T for a tile of 8 rows in shared memory, in the
+// C-fragment layout
 //   c[0], c[1] = (column g,     rows 2t, 2t + 1);  c[2], c[3] = (column g + 8, same rows).
-// The first d columns of the tile always take part, the k-steps beyond (raw features behind the
-// embedding) only when `wide` (uniform over the warp). Three independent accumulators: a
-// dependent mma.sync can issue after about 21 cycles and the pipe takes one from a warp every
-// 8, so three chains keep it fed.
+// `heads` is this lane's ldmatrix address in the tile's heads (row lane % 8, block lane / 8, see
+// ldmatrix_lane_offset), `tails` the same in its tails. NKS k-steps: d / 8 for the embedding
+// columns, one or two more for the raw features behind them (f's first layer). Three independent
+// accumulators: a dependent mma.sync can issue after about 21 cycles and the pipe takes one from
+// a warp every 8, so three chains keep it fed. The fragments of the next pair of k-steps are
+// requested before the products of this one.
+__device__ __forceinline__ int ldmatrix_lane_offset(int lane, int P) {
+    return ((lane & 7) * P + 4 * (lane >> 3)) * (int)sizeof(float);
+}
 template <int NKS>
-__device__ __forceinline__ void tile_product(const AFrag<NKS> &w, const float *buf, int P, int lane, bool wide,
-                                             float (&c)[4]) {
+__device__ __forceinline__ void tile_product(const AFrag<NKS> &w, unsigned heads, unsigned tails, float (&c)[4]) {
+    static_assert(NKD == 8 && NKS >= NKD && NKS <= NKD + 2, "four pairs of k-steps written out below, and a tail");
     float hh[4] = {0.f, 0.f, 0.f, 0.f}, hl[4] = {0.f, 0.f, 0.f, 0.f}, lh[4] = {0.f, 0.f, 0.f, 0.f};
-    const float *at = buf + (lane & 7) * P + 4 * (lane >> 3);      // row lane % 8, block lane / 8
-    const int tail = kTile * P;
-    // the fragments of the next pair of k-steps are requested before the products of this one
-    constexpr int NP = NKD / 2;
-    unsigned bh[2][4], bl[2][4];
-    ldmatrix4(bh[0], at);
-    ldmatrix4(bl[0], at + tail);
-#pragma unroll
-    for (int kp = 0; kp < NP; ++kp) {
-        if (kp + 1 < NP) {
-            ldmatrix4(bh[(kp + 1) & 1], at + 16 * (kp + 1));
-            ldmatrix4(bl[(kp + 1) & 1], at + 16 * (kp + 1) + tail);
-        }
+    auto pair = [&](int kp, const unsigned (&bh)[4], const unsigned (&bl)[4], int count) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
+            if (j >= count) break;
             const int ks = 2 * kp + j;
-            mma_tf32(lh, w.l[ks], bh[kp & 1][2 * j], bh[kp & 1][2 * j + 1]);
-            mma_tf32(hl, w.h[ks], bl[kp & 1][2 * j], bl[kp & 1][2 * j + 1]);
-            mma_tf32(hh, w.h[ks], bh[kp & 1][2 * j], bh[kp & 1][2 * j + 1]);
+            mma_tf32(lh, w.l[ks], bh[2 * j], bh[2 * j + 1]);
+            mma_tf32(hl, w.h[ks], bl[2 * j], bl[2 * j + 1]);
+            mma_tf32(hh, w.h[ks], bh[2 * j], bh[2 * j + 1]);
         }
+    };
+    unsigned bh0[4], bl0[4], bh1[4], bl1[4];
+    ldmatrix4<0>(bh0, heads);
+    ldmatrix4<0>(bl0, tails);
+    ldmatrix4<64>(bh1, heads);
+    ldmatrix4<64>(bl1, tails);
+    pair(0, bh0, bl0, 2);
+    ldmatrix4<128>(bh0, heads);
+    ldmatrix4<128>(bl0, tails);
+    pair(1, bh1, bl1, 2);
+    ldmatrix4<192>(bh1, heads);
+    ldmatrix4<192>(bl1, tails);
+    pair(2, bh0, bl0, 2);
+    if (NKS == NKD + 2) {
+        ldmatrix4<256>(bh0, heads);
+        ldmatrix4<256>(bl0, tails);
+    } else if (NKS == NKD + 1) {
+        unsigned eh[2], el[2];      // lanes 0 .. 15 give the addresses: blocks 0 and 1, as above
+        ldmatrix2<256>(eh, heads);
+        ldmatrix2<256>(el, tails);
+        bh0[0] = eh[0]; bh0[1] = eh[1];
+        bl0[0] = el[0]; bl0[1] = el[1];
     }
-    if (wide) {
-        if (NKS - NKD == 2) {
-            ldmatrix4(bh[0], at + 16 * NP);
-            ldmatrix4(bl[0], at + 16 * NP + tail);
-        } else {
-            unsigned eh[2], el[2];
-            const float *last = buf + (lane & 7) * P + 4 * ((lane >> 3) & 1) + 8 * NKD;
-            ldmatrix2(eh, last);
-            ldmatrix2(el, last + tail);
-            bh[0][0] = eh[0]; bh[0][1] = eh[1];
-            bl[0][0] = el[0]; bl[0][1] = el[1];
-        }
-#pragma unroll
-        for (int j = 0; j < NKS - NKD; ++j) {
-            const int ks = NKD + j;
-            mma_tf32(lh, w.l[ks], bh[0][2 * j], bh[0][2 * j + 1]);
-            mma_tf32(hl, w.h[ks], bl[0][2 * j], bl[0][2 * j + 1]);
-            mma_tf32(hh, w.h[ks], bh[0][2 * j], bh[0][2 * j + 1]);
-        }
-    }
+    pair(3, bh1, bl1, 2);
+    if (NKS > NKD) pair(4, bh0, bl0, NKS - NKD);
 #pragma unroll
     for (int i = 0; i < 4; ++i) c[i] = hh[i] + (hl[i] + lh[i]);
 }
@@ -324,6 +326,9 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
     float *out_ring = STAGE == 0 ? ring1 : STAGE == 1 ? ring2 : ring3;
     constexpr int in_P = STAGE == 2 ? PF : kP, out_P = STAGE == 1 ? PF : kP;
     constexpr int in_bar = kFirstBar + STAGE * kRing, out_bar = in_bar + kRing;
+    // this lane's ldmatrix address in slot 0 of the input ring, and the bytes of a tile (heads + tails)
+    const unsigned in_lane = smem_addr(in_ring) + ldmatrix_lane_offset(lane, in_P);
+    constexpr unsigned in_tile_bytes = 2 * kTile * in_P * sizeof(float);
     // The walk starts one level early, with nothing to compute: the last layer's group gathers
     // the first tiles of level 0 there and the second layer of g requests its raw features, in
     // the same code that does it between two levels (one call site each, inlined).
@@ -359,7 +364,8 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 }
                 await_tile(in_bar + slot);
                 float c[4];
-                tile_product<NKW>(w, in_ring + slot * 2 * kTile * in_P, in_P, lane, wide, c);
+                const unsigned heads = in_lane + slot * in_tile_bytes;
+                tile_product<NKW>(w, heads, heads + in_tile_bytes / 2, c);
                 const float v[4] = {fmaxf(c[0] + b_lo, 0.f), fmaxf(c[1] + b_lo, 0.f), fmaxf(c[2] + b_hi, 0.f),
                                     fmaxf(c[3] + b_hi, 0.f)};      // (row 2t, col), (2t + 1, col), (2t, col + 8), (2t + 1, col + 8)
                 if (STAGE != 3) {
