@@ -118,7 +118,8 @@ struct AFrag {
 
 // c = (this warp's 16 columns of W)^T x (tile)^T for a tile of 8 rows in shared memory, in the
 // C-fragment layout
-//   c[0], c[1] = (column g,     rows 2t, 2t + 1);  c[2], c[3] = (column g + 8, same rows).
+//   c[0], c[1] = (column g,     rows 2t, 2t + 1);  c[2], c[3] = (column g + 8, same rows),
+// plus the bias of the two columns (the accumulators start from it).
 // `heads` is this lane's ldmatrix address in the tile's heads (row lane % 8, block lane / 8, see
 // ldmatrix_lane_offset), `tails` the same in its tails. NKS k-steps: d / 8 for the embedding
 // columns, one or two more for the raw features behind them (f's first layer). Three independent
@@ -129,9 +130,10 @@ __device__ __forceinline__ int ldmatrix_lane_offset(int lane, int P) {
     return ((lane & 7) * P + 4 * (lane >> 3)) * (int)sizeof(float);
 }
 template <int NKS>
-__device__ __forceinline__ void tile_product(const AFrag<NKS> &w, unsigned heads, unsigned tails, float (&c)[4]) {
+__device__ __forceinline__ void tile_product(const AFrag<NKS> &w, unsigned heads, unsigned tails, float b_lo, float b_hi,
+                                             float (&c)[4]) {
     static_assert(NKD == 8 && NKS >= NKD && NKS <= NKD + 2, "four pairs of k-steps written out below, and a tail");
-    float hh[4] = {0.f, 0.f, 0.f, 0.f}, hl[4] = {0.f, 0.f, 0.f, 0.f}, lh[4] = {0.f, 0.f, 0.f, 0.f};
+    float hh[4] = {b_lo, b_lo, b_hi, b_hi}, hl[4] = {0.f, 0.f, 0.f, 0.f}, lh[4] = {0.f, 0.f, 0.f, 0.f};     // bias: columns g, g + 8
     auto pair = [&](int kp, const unsigned (&bh)[4], const unsigned (&bl)[4], int count) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
@@ -260,8 +262,8 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
     __syncthreads();              // schedule staged
     dependency_wait();            // the raw features may come from a kernel that is still running
 
-    unsigned tc = 0;              // tiles this warp has taken from its input ring
-    unsigned tg = 0;              // last layer: tiles gathered
+    int slot = 0;                 // ring slot of the tile this warp takes next (tiles taken so far modulo kRing)
+    int g_slot = 0;               // last layer: ring slot of the tile gathered next
     int g_level = 0, g_j = 0;     //             the next tile to gather
 
     // Last layer: sum of the neighbours' messages of tile j of a level, split, into the first
@@ -284,14 +286,14 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 acc.w += v.w;
             }
         }
-        float *out = ring0 + (tg % kRing) * 2 * kTail + rr * kP + c4;
+        float *out = ring0 + g_slot * 2 * kTail + rr * kP + c4;
         const float4 head = make_float4(tf32_round(acc.x), tf32_round(acc.y), tf32_round(acc.z), tf32_round(acc.w));
         *reinterpret_cast<float4 *>(out) = head;
         *reinterpret_cast<float4 *>(out + kTail) =
             make_float4(tf32_round(acc.x - head.x), tf32_round(acc.y - head.y), tf32_round(acc.z - head.z),
                         tf32_round(acc.w - head.w));
-        tile_ready(kFirstBar + tg % kRing);
-        ++tg;
+        tile_ready(kFirstBar + g_slot);
+        g_slot = g_slot == kRing - 1 ? 0 : g_slot + 1;
     };
     // Second layer of g: the raw features of a level, one level ahead. Every thread fetches exactly
     // the word it will itself copy into each tile, so its own wait is all the synchronisation needed.
@@ -341,7 +343,6 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
 #pragma unroll 1
         for (int j = 0; j < n_tiles; ++j) {
             if (level >= 0) {
-                const int slot = tc % kRing;
                 // ---- before the tile arrives: whatever does not depend on it
                 float *dst[2] = {nullptr, nullptr};             // second layers: where rows 2t, 2t + 1 go (h_v / m_u)
                 if (second) {
@@ -365,9 +366,9 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 await_tile(in_bar + slot);
                 float c[4];
                 const unsigned heads = in_lane + slot * in_tile_bytes;
-                tile_product<NKW>(w, heads, heads + in_tile_bytes / 2, c);
-                const float v[4] = {fmaxf(c[0] + b_lo, 0.f), fmaxf(c[1] + b_lo, 0.f), fmaxf(c[2] + b_hi, 0.f),
-                                    fmaxf(c[3] + b_hi, 0.f)};      // (row 2t, col), (2t + 1, col), (2t, col + 8), (2t + 1, col + 8)
+                tile_product<NKW>(w, heads, heads + in_tile_bytes / 2, b_lo, b_hi, c);
+                // (row 2t, col), (2t + 1, col), (2t, col + 8), (2t + 1, col + 8)
+                const float v[4] = {fmaxf(c[0], 0.f), fmaxf(c[1], 0.f), fmaxf(c[2], 0.f), fmaxf(c[3], 0.f)};
                 if (STAGE != 3) {
                     float *out = out_ring + slot * 2 * kTile * out_P + 2 * t * out_P + col;
                     const int tail = kTile * out_P;
@@ -385,7 +386,7 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                             dst[i][8] = v[2 + i];
                         }
                 }
-                ++tc;
+                slot = slot == kRing - 1 ? 0 : slot + 1;
             }
             if (STAGE == 3) {
                 // Sums for the tiles ahead. Inside a level: one more tile for the one just taken
