@@ -165,14 +165,13 @@ typedef struct {
                                   d = 64 otherwise takes */
 #define PLACETO_TENSOR 32u     /* use the tensor-core kernel of step 2 that gives every block whole 16-row
                                   tiles (all warps on one layer at a time) wherever it applies (d = 32 or
-                                  64), also where the library would pick another one */
+                                  64); the library itself picks other kernels there */
 #define PLACETO_TCGEN05 64u    /* d = 64: take the kernel built on tcgen05.mma with accumulators in tensor
                                   memory instead of the warp-level (mma.sync) tensor-core kernel that is
                                   the default there (measured slower at the configured batch sizes) */
 #define PLACETO_PIPELINE 128u  /* d = 64: take the kernel that runs the four layers of g and f as a pipeline
-                                  (a group of warps per layer, tiles of eight rows), also for batches so
-                                  large that the library would pick the 16-row-tile kernel (the default
-                                  up to eight states per thread block) */
+                                  (a group of warps per layer, tiles of eight rows). It is what the
+                                  library picks at d = 64 anyway; the flag pins the choice. */
 
 typedef enum {
     PLACETO_CALL_EMBED = 0,       /* placeto_embed_forward */

@@ -219,7 +219,7 @@ placeto_status run_embed(const placeto_graph *g, const placeto_weights *w, const
         cudaError_t e = launch_embed_tc(a, g->info, stream, after_own_kernel);
         if (e != cudaErrorNotSupported) return cuda_status(e);
     }
-    // d = 64: the pipeline of layers where it is the faster one (or asked for), if it fits
+    // d = 64: the pipeline of layers, if it fits
     if (!(flags & (PLACETO_GENERIC | PLACETO_FMA_ONLY | PLACETO_TENSOR)) && schedule == PLACETO_SLICED &&
         ((flags & PLACETO_PIPELINE) ? embed_pipe_applicable(a) : embed_pipe_preferred(a, g->info))) {
         cudaError_t e = launch_embed_pipe(a, g->info, stream, after_own_kernel);

@@ -444,6 +444,10 @@ cudaError_t launch(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream
     };
     while (p.S > 1 && need(p.S) > budget) --p.S;
     if (need(p.S) > budget) return cudaErrorNotSupported;
+    // Shared memory may force more slices than one wave of blocks holds: spread the batch evenly over
+    // the waves it then takes (two full waves finish before one full wave and a ragged one of larger slices)
+    const int waves = ((a.B + p.S - 1) / p.S + want - 1) / want;
+    p.S = std::min(p.S, (a.B + want * waves - 1) / (want * waves));
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.x_floats = x_floats(p.S);
     p.smem_bytes = need(p.S);
@@ -465,14 +469,9 @@ bool embed_pipe_applicable(const EmbedArgs &a) {
 }
 
 // Measured on B200 on the NASNet-shaped graph (n = 2130, 744 levels), pipeline against the
-// 16-row-tile kernel: 1.36 against 1.72 ms at B = 64, 1.91 / 2.09 at 256, 2.81 / 2.94 at 512, 4.91 /
-// 4.92 at 1024, 14.8 / 9.2 at 2048. The pipeline wins while a level has a few tiles of eight rows
-// (the layers of one tile overlap with those of the next); with many rows per level both are bound
-// by throughput, where the pipeline issues more instructions per row.
-bool embed_pipe_preferred(const EmbedArgs &a, const DeviceInfo &di) {
-    const int blocks = std::max(1, di.sm_count / 2);
-    return embed_pipe_applicable(a) && (a.B + blocks - 1) / blocks <= 8;
-}
+// 16-row-tile kernel, ms: 0.90 / 1.72 at B = 64, 1.37 / 2.09 at 256, 2.10 / 2.94 at 512, 3.75 / 4.92 at
+// 1024, 7.48 / 9.19 at 2048, 14.9 / 18.2 at 4096: the pipeline is taken wherever it applies.
+bool embed_pipe_preferred(const EmbedArgs &a, const DeviceInfo &) { return embed_pipe_applicable(a); }
 
 cudaError_t launch_embed_pipe(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap) {
     return a.F <= 8 ? launch<9>(a, di, stream, overlap) : launch<10>(a, di, stream, overlap);

@@ -344,7 +344,7 @@ cudaError_t launch_embed_mma(const EmbedArgs &a, const DeviceInfo &di, cudaStrea
 // tiles of eight rows handed from layer to layer through shared memory). cudaErrorNotSupported when
 // the schedule and the message slots do not fit in shared memory.
 bool embed_pipe_applicable(const EmbedArgs &a);
-bool embed_pipe_preferred(const EmbedArgs &a, const DeviceInfo &di);   // applicable and faster than the tile kernel
+bool embed_pipe_preferred(const EmbedArgs &a, const DeviceInfo &di);   // where the library picks it
 cudaError_t launch_embed_pipe(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream, bool overlap = false);
 
 // embed_tc.cu: d = 64 on tcgen05 tensor cores with accumulators in tensor memory (TF32 head + tail
