@@ -295,7 +295,7 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
         tile_ready(kFirstBar + g_slot);
         g_slot = g_slot == kRing - 1 ? 0 : g_slot + 1;
     };
-    // Second layer of g: the raw features of a level, one level ahead. Every thread fetches exactly
+    // First layer of g: the raw features of a level, one level ahead. Every thread fetches exactly
     // the word it will itself copy into each tile, so its own wait is all the synchronisation needed.
     const int x_row = gt / XC, x_col = gt - x_row * XC;          // gt < kTile * XC: a word of every tile
     const bool x_mine = gt < kTile * XC;
@@ -332,14 +332,14 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
     const unsigned in_lane = smem_addr(in_ring) + ldmatrix_lane_offset(lane, in_P);
     constexpr unsigned in_tile_bytes = 2 * kTile * in_P * sizeof(float);
     // The walk starts one level early, with nothing to compute: the last layer's group gathers
-    // the first tiles of level 0 there and the second layer of g requests its raw features, in
+    // the first tiles of level 0 there and the first layer of g requests its raw features, in
     // the same code that does it between two levels (one call site each, inlined).
 #pragma unroll 1
     for (int level = -1; level < lv.n_levels; ++level) {
         const int p0 = level < 0 ? 0 : level_ptr[level], rows = level < 0 ? 0 : (level_ptr[level + 1] - p0) * nb;
         const int n_tiles = level < 0 ? (STAGE == 3 ? 1 : 0) : (rows + kTile - 1) / kTile;
         const float *xs = xstage + (size_t)(level & 1) * p.x_floats;
-        if (STAGE == 1) __pipeline_wait_prior(0);          // this level's raw features: requested a level ago
+        if (STAGE == 0) __pipeline_wait_prior(0);          // this level's raw features: requested a level ago
 #pragma unroll 1
         for (int j = 0; j < n_tiles; ++j) {
             if (level >= 0) {
@@ -356,12 +356,14 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                             else if (m.z >= 0) dst[i] = msg + ((size_t)m.z * S + (r - q * nb)) * kP + col;
                         }
                     }
-                    if (STAGE == 1 && x_mine) {
-                        // the raw features (zero padded) behind the d embedding columns of the output tile
-                        const int r = kTile * j + x_row;
-                        store_split(out_ring + slot * 2 * kTile * PF + x_row * PF + kD + x_col, kTile * PF,
-                                    (r < rows && x_col < F) ? xs[r * F + x_col] : 0.f);
-                    }
+                }
+                if (STAGE == 0 && x_mine) {
+                    // The raw features (zero padded) behind the d embedding columns of the tile that f's
+                    // first layer will read, two rings on: its slot is free (at most kRing tiles are
+                    // in flight), and this group has the lightest layer.
+                    const int r = kTile * j + x_row;
+                    store_split(ring2 + slot * 2 * kTile * PF + x_row * PF + kD + x_col, kTile * PF,
+                                (r < rows && x_col < F) ? xs[r * F + x_col] : 0.f);
                 }
                 await_tile(in_bar + slot);
                 float c[4];
@@ -405,7 +407,7 @@ embed_pipe_kernel(const EmbedArgs a, const PipePlan p) {
                 for (; g_j < upto; ++g_j) gather(g_level, g_j);
             }
         }
-        if (STAGE == 1 && level + 1 < lv.n_levels) prefetch(level + 1);      // the other buffer: its level is done
+        if (STAGE == 0 && level + 1 < lv.n_levels) prefetch(level + 1);      // the other buffer: its level is done
     }
     };
     switch (stage) {
