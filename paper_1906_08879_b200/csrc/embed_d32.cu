@@ -343,6 +343,11 @@ bool plan_d32(const EmbedArgs &a, const DeviceInfo &di, D32Plan *out) {
     // narrower slices when the shared memory does not fit (more blocks: they queue up)
     while (p.S > 1 && need(p.S) > budget) --p.S;
     if (need(p.S) > budget) return false;
+    // more slices than one wave of blocks: spread the batch evenly over the waves it takes
+    {
+        const int waves = ((a.B + p.S - 1) / p.S + want - 1) / want;
+        p.S = std::min(p.S, (a.B + want * waves - 1) / (want * waves));
+    }
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.x_floats = x_floats(p.S);
     p.smem_bytes = need(p.S);

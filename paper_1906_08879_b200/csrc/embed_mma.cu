@@ -364,6 +364,11 @@ cudaError_t launch(const EmbedArgs &a, const DeviceInfo &di, cudaStream_t stream
     };
     while (p.S > 1 && need(p.S) > budget) --p.S;
     if (need(p.S) > budget) return cudaErrorNotSupported;
+    // more slices than one wave of blocks: spread the batch evenly over the waves it takes
+    {
+        const int waves = ((a.B + p.S - 1) / p.S + want - 1) / want;
+        p.S = std::min(p.S, (a.B + want * waves - 1) / (want * waves));
+    }
     p.n_slices = (a.B + p.S - 1) / p.S;
     p.x_floats = x_floats(p.S);
     p.smem_bytes = need(p.S);
